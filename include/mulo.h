@@ -1,0 +1,210 @@
+/*
+ * mulo.h -- C ABI of the B200 (sm_100a) draft-and-verify round of Multi-Scale
+ * Local Speculative Decoding (MuLo-SD) for autoregressive image generation.
+ *
+ * One speculative round over an H x W grid of image tokens, for B independent
+ * images, given the target model's logits at every position and the drafter's
+ * logits on the (H/r) x (W/r) low-resolution grid:
+ *
+ *   up-sample draft tokens and draft distributions to the target grid
+ *   -> target / draft probabilities over the vocabulary (CFG, temperature, top-k)
+ *   -> acceptance test  u < min(1, P / q(x~))        (Sec. 3.1, Eq. 1 and Eq. 3)
+ *   -> rejection mask R_T, first rejection t_0       (Sec. 3.3)
+ *   -> local expansion R_X                           (Sec. 3.3, Eq. 6-7)
+ *   -> parallel inverse-CDF redraw of R_X            (Eq. 2; Algorithm 1 Step 6)
+ *
+ * Conventions for every call
+ *   - All tensor arguments are DEVICE pointers to caller-owned, contiguous,
+ *     row-major memory, 16-byte aligned, unless the name says "host".  The
+ *     library never allocates or frees device memory; scratch space is the
+ *     workspace the caller hands to mulo_set_workspace.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls validate their arguments on the host, enqueue kernels on the stream
+ *     and return; outputs are defined once the stream has been synchronised.
+ *   - Errors are return codes.  An invalid argument is detected before anything
+ *     is launched.  Kernels never trap; contract violations they can see (a
+ *     draft token with zero draft probability, a token id outside [0, V)) set a
+ *     bit that mulo_poll_device_status reports.
+ *   - Positions are raster indices t = i * W + j.  Bit masks hold one bit per
+ *     position: bit (j % 32) of word (b * H + i) * ceil(W / 32) + j / 32.
+ *   - Logit tensors share one dtype (fp32, or bf16 as raw 16-bit patterns) and
+ *     must be finite.  V must be a multiple of 8 and at most 65536.
+ *   - Uniform random numbers: Philox4x32-10 with key (seed low word, seed high
+ *     word) and counter (position t, image b + image_offset, round, 0); output
+ *     word 0 drives the acceptance test, word 1 the residual draw, word 2 the
+ *     draw from the target distribution; u = (word >> 8) * 2^-24.
+ */
+#ifndef MULO_H_
+#define MULO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mulo_ctx mulo_ctx; /* opaque; one per device and host thread */
+
+typedef enum {
+  MULO_OK = 0,
+  MULO_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, bad shape or parameter        */
+  MULO_ERR_UNSUPPORTED = 2, /* valid but outside what the kernels handle (see limits)   */
+  MULO_ERR_WORKSPACE = 3,   /* no workspace set, or too small for these parameters      */
+  MULO_ERR_CUDA = 4,        /* a CUDA runtime call failed (also: no usable device)      */
+  MULO_ERR_TIMEOUT = 5      /* reserved for bounded device-side waits; unused today     */
+} mulo_status;
+
+typedef enum { MULO_F32 = 0, MULO_BF16 = 1 } mulo_dtype;
+
+typedef enum {
+  MULO_ACCEPT_RATIO = 0,    /* Eq. 1 with Eq. 3's pooled numerator: u < min(1, P/q(x~))  */
+  MULO_ACCEPT_THRESHOLD = 1 /* Eq. 5: accept iff pooled target mass P >= tau (no q, no u) */
+} mulo_accept_mode;
+
+typedef enum {
+  MULO_RESAMPLE_MIXED = 0,        /* rejected positions: residual of Eq. 2; the rest of R_X:
+                                     the target distribution (Algorithm 1 Step 6)            */
+  MULO_RESAMPLE_RESIDUAL_ALL = 1, /* every position of R_X from the residual                  */
+  MULO_RESAMPLE_TARGET_ALL = 2,   /* every position of R_X from the target distribution       */
+  MULO_RESAMPLE_ISOLATED_RESIDUAL = 3 /* residual only for a rejected position that no other
+                                     rejection would have swept in; target distribution for
+                                     the rest of R_X (exact for independent draft tokens)   */
+} mulo_resample_mode;
+
+/* device status bits (mulo_poll_device_status) */
+#define MULO_DEV_ZERO_DRAFT_PROB 1u /* some draft token had q(x~) == 0                    */
+#define MULO_DEV_BAD_TOKEN 2u       /* some token / neighbour id was outside [0, V)        */
+#define MULO_DEV_DENSE_FALLBACK 4u  /* informational: a row left the fast top-k path       */
+
+typedef struct mulo_params {
+  int32_t B, H, W;       /* images, target grid; the draft grid is (H/r) x (W/r)            */
+  int32_t V;             /* vocabulary size: multiple of 8, <= 65536                         */
+  int32_t r;             /* resolution ratio s_p / s_q >= 1; H % r == 0 and W % r == 0       */
+  int32_t logit_dtype;   /* mulo_dtype of all three logit tensors                            */
+  float temperature;     /* > 0; logits are multiplied by fp32(1 / temperature)              */
+  int32_t top_k;         /* <= 0 or >= V: off.  Otherwise keep every entry >= the k-th
+                            largest value of the row (ties kept); same k for target/draft   */
+  float cfg_scale;       /* s of l = l_u + s (l_c - l_u); used iff an unconditional tensor
+                            is passed                                                        */
+  int32_t accept_mode;   /* mulo_accept_mode                                                 */
+  float tau;             /* Eq. 5 threshold (MULO_ACCEPT_THRESHOLD only)                     */
+  int32_t pool_k;        /* codebook neighbourhood size k of Eq. 3; <= 1 turns pooling off;
+                            at most 2048                                                     */
+  float pool_delta;      /* delta of Eq. 4: the pooled neighbours may add < delta of mass    */
+  int32_t radius;        /* l of Eq. 6, 0 <= l <= 31; l rounds of 3x3 growth                 */
+  int32_t clip_before_first; /* non-zero: keep Eq. 6's clause u >= t_0                       */
+  int32_t resample_mode; /* mulo_resample_mode                                               */
+  uint64_t seed;         /* Philox key                                                       */
+  uint32_t round;        /* speculative round index (Philox counter word 2)                  */
+  uint32_t image_offset; /* added to the image index b in Philox counter word 1, so that a
+                            batch split over several calls or devices draws the same numbers */
+} mulo_params;
+
+/* ---- context, workspace, diagnostics (no counterpart in the paper) ------------------- */
+
+/* Creates a context bound to CUDA device `device` (queries its limits, raises the
+ * kernels' dynamic shared-memory caps).  Returns MULO_ERR_CUDA if the device cannot be
+ * used.  The context is host memory owned by the library until mulo_destroy. */
+mulo_status mulo_create(mulo_ctx** out, int device);
+void mulo_destroy(mulo_ctx* ctx);
+const char* mulo_status_string(mulo_status s);
+
+/* Bytes of device scratch that calls with these parameters need (status word, per-position
+ * accept flags and candidate tokens). */
+mulo_status mulo_workspace_bytes(const mulo_params* p, size_t* bytes);
+/* Hands the library a caller-owned device buffer (256-byte aligned).  It must stay valid
+ * and must not be shared by calls that overlap on the device.  The first 256 bytes hold
+ * the device status word; this call clears it (on the default stream, synchronously). */
+mulo_status mulo_set_workspace(mulo_ctx* ctx, void* dev_ptr, size_t bytes);
+/* Synchronises `stream`, reads and clears the device status bits (MULO_DEV_*). */
+mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags);
+/* Number of kernels this context has launched so far. */
+mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
+
+/* ---- the four stages ------------------------------------------------------------------ */
+
+/* Step 2 of the pipeline (Sec. 3.2: x~ = U_r(y~), r^2 times as many tokens) with the
+ * nearest-neighbour stand-in for U_r, plus the part of the pooled acceptance rule (Eq. 3)
+ * that needs only the drafter: per low-res cell the draft row's top-k threshold theta_q,
+ * maximum m_q and partition sum Z_q (so that q(x) = [z >= theta_q] exp(z - m_q) / Z_q),
+ * and q(x~) at every target position.
+ *   draft_logits_lo [B, h, w, V]   in
+ *   draft_tok_lo    [B, h, w]      in   int32 token ids
+ *   nn              [V, pool_k]    in   uint16; unused here, may be NULL
+ *   draft_tok_hi    [B, H, W]      out  x~[b,i,j] = y~[b,i/r,j/r]
+ *   draft_stats_lo  [B, h, w, 4]   out  fp32 (theta_q, m_q, Z_q high part, Z_q low part):
+ *                                       Z_q = hi + lo; theta_q = -inf if top-k is off
+ *   q_tok_hi        [B, H, W]      out  fp32 q(x~)                                        */
+mulo_status mulo_upsample_pool(mulo_ctx* ctx, const mulo_params* p, const void* draft_logits_lo,
+                               const int32_t* draft_tok_lo, const uint16_t* nn,
+                               int32_t* draft_tok_hi, float* draft_stats_lo, float* q_tok_hi,
+                               void* stream);
+
+/* Steps 3-4: target probabilities (CFG mix l_u + s (l_c - l_u), temperature, top-k, softmax;
+ * Supp. "Sampling"), pooled mass P over A_{k,delta}(x~) (Eq. 3-4; Algorithm 1), and the
+ * acceptance decision (Eq. 1, or Eq. 5 in threshold mode).
+ *   tgt_cond, tgt_uncond [B, H, W, V]  in   (tgt_uncond may be NULL: no CFG)
+ *   draft_logits_lo, draft_stats_lo, draft_tok_hi, nn   in   as above (nn required iff pool_k > 1;
+ *                                      nn[x][0] must be x, the rest distinct and != x)
+ *   p_tok, q_tok, accept_prob [B, H, W] out  fp32 p(x~), q(x~), min(1, P/q(x~)) (or P in threshold mode)
+ *   reject_bits  [B, H, ceil(W/32)]    out  uint32, 1 = rejected (R_T)
+ *   n_reject     [B]                   out  |R_T|
+ *   first_reject [B]                   out  t_0, or H*W if nothing was rejected
+ * Needs the workspace. */
+mulo_status mulo_verify(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond,
+                        const void* tgt_uncond, const void* draft_logits_lo,
+                        const float* draft_stats_lo, const int32_t* draft_tok_hi,
+                        const uint16_t* nn, float* p_tok, float* q_tok, float* accept_prob,
+                        uint32_t* reject_bits, int32_t* n_reject, int32_t* first_reject,
+                        void* stream);
+
+/* Step 5: R_X = union over rejected t of N(t, l), N(t, l) = {u : |i_u - i_t| <= l,
+ * |j_u - j_t| <= l, u >= t_0} (Eq. 6-7).
+ *   reject_bits, first_reject   in
+ *   expand_bits [B, H, ceil(W/32)]  out   n_expand [B]  out  |R_X|                        */
+mulo_status mulo_local_reject_expand(mulo_ctx* ctx, const mulo_params* p,
+                                     const uint32_t* reject_bits, const int32_t* first_reject,
+                                     uint32_t* expand_bits, int32_t* n_expand, void* stream);
+
+/* Step 6 on given logits: every position of R_X is redrawn in parallel by inverse CDF over
+ * w(x) = max(0, p'(x) - lambda q(x)) in ascending token id, lambda = 1 (Eq. 2) or 0
+ * (Algorithm 1 Step 6) as resample_mode says; p' is p with the pooled mass moved onto x~.
+ * A residual without mass falls back to lambda = 0.  Positions outside R_X keep x~.
+ *   out_tok [B, H, W]  out  int32                                                         */
+mulo_status mulo_resample(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond,
+                          const void* tgt_uncond, const void* draft_logits_lo,
+                          const float* draft_stats_lo, const int32_t* draft_tok_hi,
+                          const uint16_t* nn, const uint32_t* reject_bits,
+                          const uint32_t* expand_bits, int32_t* out_tok, void* stream);
+
+/* ---- the fused round ------------------------------------------------------------------- */
+
+/* The four stages in one pass: every logit row is read from HBM once.  Results are those
+ * of mulo_upsample_pool -> mulo_verify -> mulo_local_reject_expand -> mulo_resample.
+ *   p_tok, q_tok, accept_prob may be NULL (skipped).  Needs the workspace. */
+mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond,
+                       const void* tgt_uncond, const void* draft_logits_lo,
+                       const int32_t* draft_tok_lo, const uint16_t* nn, int32_t* out_tok,
+                       uint32_t* reject_bits, uint32_t* expand_bits, float* p_tok, float* q_tok,
+                       float* accept_prob, int32_t* n_reject, int32_t* n_expand,
+                       int32_t* first_reject, void* stream);
+
+/* mulo_round for callers whose tensors live in HOST memory (pinned memory copies fastest):
+ * copies the inputs into `arena` (caller-owned device memory of at least
+ * mulo_round_host_arena_bytes, 256-byte aligned; it also serves as the workspace, replacing
+ * any set before), runs the round, copies the results back and synchronises `stream`
+ * before returning.  All tensor arguments are HOST pointers; optional ones may be NULL. */
+mulo_status mulo_round_host_arena_bytes(const mulo_params* p, int has_uncond, size_t* bytes);
+mulo_status mulo_round_host(mulo_ctx* ctx, const mulo_params* p, void* arena, size_t arena_bytes,
+                            const void* tgt_cond, const void* tgt_uncond,
+                            const void* draft_logits_lo, const int32_t* draft_tok_lo,
+                            const uint16_t* nn, int32_t* out_tok, uint32_t* reject_bits,
+                            uint32_t* expand_bits, float* p_tok, float* q_tok,
+                            float* accept_prob, int32_t* n_reject, int32_t* n_expand,
+                            int32_t* first_reject, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MULO_H_ */

@@ -1,0 +1,792 @@
+// libmulo: kernels and C ABI of the MuLo-SD draft-and-verify round (sm_100a).
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/mulo.h"
+#include "mulo_dense.cuh"
+
+using namespace mulo;
+
+// ============================================================== row kernels
+
+struct RowKernelArgs {
+  DevParams P;
+  const char* cond;
+  const char* uncond;
+  const char* draft;
+  const int32_t* draft_tok_lo;   // fused / upsample: [B,h,w]
+  const int32_t* draft_tok_hi;   // unfused verify / resample: [B,H,W]
+  const float* stats_in;         // unfused: [B,h,w,4]
+  const uint16_t* nn;
+  const uint32_t* reject_bits;   // resample stage
+  const uint32_t* expand_bits;   // resample stage
+  // outputs
+  float* p_tok;
+  float* q_tok;
+  float* accept_prob;
+  uint8_t* flags;                // workspace: 1 = rejected
+  int32_t* cand_res;             // workspace
+  int32_t* cand_tgt;             // workspace
+  int32_t* out_tok;              // resample stage
+  int32_t* tok_hi_out;           // upsample stage
+  float* stats_out;              // upsample stage
+  float* q_tok_hi_out;           // upsample stage
+  uint32_t* dev_status;
+};
+
+__device__ __forceinline__ RowSrc target_row(const RowKernelArgs& a, size_t row) {
+  const size_t bytes = (size_t)a.P.V * (a.P.bf16 ? 2 : 4);
+  RowSrc r;
+  r.cond = a.cond + row * bytes;
+  r.uncond = a.uncond ? a.uncond + row * bytes : nullptr;
+  r.s = a.P.cfg_scale;
+  r.invT = a.P.invT;
+  r.V = a.P.V;
+  r.bf16 = a.P.bf16;
+  return r;
+}
+__device__ __forceinline__ RowSrc draft_row(const RowKernelArgs& a, size_t cell) {
+  const size_t bytes = (size_t)a.P.V * (a.P.bf16 ? 2 : 4);
+  RowSrc r;
+  r.cond = a.draft + cell * bytes;
+  r.uncond = nullptr;
+  r.s = 0.f;
+  r.invT = a.P.invT;
+  r.V = a.P.V;
+  r.bf16 = a.P.bf16;
+  return r;
+}
+
+__device__ __forceinline__ PoolSmem carve_pool(const DevParams& P, unsigned char* dyn) {
+  PoolSmem ps;
+  ps.pn = reinterpret_cast<double*>(dyn);
+  ps.bitmap = reinterpret_cast<uint32_t*>(dyn + (size_t)max(P.pool_k, 1) * sizeof(double));
+  return ps;
+}
+
+__device__ __forceinline__ int checked_token(int tok, int V, uint32_t* dev_status) {
+  if (tok < 0 || tok >= V) {
+    if (threadIdx.x == 0) atomicOr(dev_status, MULO_DEV_BAD_TOKEN);
+    tok = min(max(tok, 0), V - 1);
+  }
+  return tok;
+}
+
+// Which draws does a visit need once its accept bit is known (fused round)?
+__device__ __forceinline__ int draws_for(int mode, int accepted) {
+  int d = 0;
+  if (mode == MULO_RESAMPLE_RESIDUAL_ALL || (!accepted && mode != MULO_RESAMPLE_TARGET_ALL)) d |= kDrawResidual;
+  if (mode == MULO_RESAMPLE_TARGET_ALL || (accepted && mode != MULO_RESAMPLE_RESIDUAL_ALL) ||
+      (!accepted && mode == MULO_RESAMPLE_ISOLATED_RESIDUAL))
+    d |= kDrawTarget;
+  return d;
+}
+
+// mulo_upsample_pool: one CTA per low-res cell.
+__global__ void __launch_bounds__(kThreads) k_upsample_pool(RowKernelArgs a) {
+  __shared__ BlockScratch bs;
+  const DevParams& P = a.P;
+  const int cell = blockIdx.x;   // b*h*w + ca*w + cc
+  const int b = cell / (P.h * P.w), rem = cell % (P.h * P.w), ca = rem / P.w, cc = rem % P.w;
+  RowSrc qr = draft_row(a, cell);
+  RowStats sq;
+  dense_row_stats(qr, P.top_k, bs, sq.theta, sq.m, sq.Z);
+  if (threadIdx.x == 0) {
+    const int tok = checked_token(a.draft_tok_lo[cell], P.V, a.dev_status);
+    const float Zhi = (float)sq.Z, Zlo = (float)(sq.Z - (double)Zhi);
+    a.stats_out[(size_t)cell * 4 + 0] = sq.theta;
+    a.stats_out[(size_t)cell * 4 + 1] = sq.m;
+    a.stats_out[(size_t)cell * 4 + 2] = Zhi;
+    a.stats_out[(size_t)cell * 4 + 3] = Zlo;
+    float zq = load1(qr, tok);
+    double q = (zq >= sq.theta) ? exp((double)zq - (double)sq.m) / ((double)Zhi + (double)Zlo) : 0.0;
+    for (int di = 0; di < P.r; ++di)
+      for (int dj = 0; dj < P.r; ++dj) {
+        size_t t = ((size_t)b * P.H + (size_t)ca * P.r + di) * P.W + (size_t)cc * P.r + dj;
+        a.tok_hi_out[t] = a.draft_tok_lo[cell];
+        a.q_tok_hi_out[t] = (float)q;
+      }
+  }
+}
+
+// mulo_verify (FUSED = false): one CTA per target position, draft statistics given.
+// mulo_round  (FUSED = true):  one CTA per low-res cell: draft statistics, then its
+// r*r children; accept flags and candidate draws go to the workspace.
+template <bool FUSED>
+__global__ void __launch_bounds__(kThreads) k_verify_rows(RowKernelArgs a) {
+  __shared__ BlockScratch bs;
+  extern __shared__ __align__(16) unsigned char dyn[];
+  const DevParams& P = a.P;
+  PoolSmem ps = carve_pool(P, dyn);
+  const int N = P.H * P.W;
+  if (FUSED) {
+    const int cell = blockIdx.x;
+    const int b = cell / (P.h * P.w), rem = cell % (P.h * P.w), ca = rem / P.w, cc = rem % P.w;
+    RowSrc qr = draft_row(a, cell);
+    RowStats sq;
+    dense_row_stats(qr, P.top_k, bs, sq.theta, sq.m, sq.Z);
+    {   // the unfused path stores Z_q as an fp32 (hi, lo) pair; keep both paths identical
+      const float Zhi = (float)sq.Z, Zlo = (float)(sq.Z - (double)Zhi);
+      sq.Z = (double)Zhi + (double)Zlo;
+    }
+    const int tok = checked_token(a.draft_tok_lo[cell], P.V, a.dev_status);
+    for (int di = 0; di < P.r; ++di)
+      for (int dj = 0; dj < P.r; ++dj) {
+        const int t = (ca * P.r + di) * P.W + cc * P.r + dj;
+        const size_t g = (size_t)b * N + t;
+        RowSrc tr = target_row(a, g);
+        PositionOut o;
+        const int mode = P.resample_mode;
+        dense_position(P, tr, qr, sq, tok, a.nn, (uint32_t)b + P.image_offset, (uint32_t)t, true, 0,
+                       [mode](int acc) { return draws_for(mode, acc); }, bs, ps, a.dev_status, o);
+        if (threadIdx.x == 0) {
+          a.flags[g] = o.accepted ? 0 : 1;
+          a.cand_res[g] = o.tok_residual;
+          a.cand_tgt[g] = o.tok_target;
+          if (a.p_tok) a.p_tok[g] = o.p_tok;
+          if (a.q_tok) a.q_tok[g] = o.q_tok;
+          if (a.accept_prob) a.accept_prob[g] = o.accept_prob;
+        }
+        __syncthreads();
+      }
+  } else {
+    const size_t g = blockIdx.x;
+    const int b = (int)(g / N), t = (int)(g % N), i = t / P.W, j = t % P.W;
+    const size_t cell = ((size_t)b * P.h + i / P.r) * P.w + j / P.r;
+    RowSrc qr = draft_row(a, cell);
+    RowStats sq;
+    sq.theta = a.stats_in[cell * 4 + 0];
+    sq.m = a.stats_in[cell * 4 + 1];
+    sq.Z = (double)a.stats_in[cell * 4 + 2] + (double)a.stats_in[cell * 4 + 3];
+    const int tok = checked_token(a.draft_tok_hi[g], P.V, a.dev_status);
+    RowSrc tr = target_row(a, g);
+    PositionOut o;
+    dense_position(P, tr, qr, sq, tok, a.nn, (uint32_t)b + P.image_offset, (uint32_t)t, true, 0,
+                   [](int) { return (int)kDrawNone; }, bs, ps, a.dev_status, o);
+    if (threadIdx.x == 0) {
+      a.flags[g] = o.accepted ? 0 : 1;
+      a.p_tok[g] = o.p_tok;
+      a.q_tok[g] = o.q_tok;
+      a.accept_prob[g] = o.accept_prob;
+    }
+  }
+}
+
+__device__ __forceinline__ int get_bit(const uint32_t* bits, int Ww, int H, int b, int i, int j) {
+  return (bits[((size_t)b * H + i) * Ww + (j >> 5)] >> (j & 31)) & 1u;
+}
+
+// Would position (i,j), if it had been accepted, have been swept into R_X by
+// another rejection?  (some other rejected position within radius l, and -- with
+// clipping -- (i,j) is not the image's first rejection)
+__device__ __forceinline__ bool covered_by_other(const uint32_t* rej, int Ww, int H, int W, int b, int i,
+                                                 int j, int l, int clip, int t0) {
+  if (clip && i * W + j == t0) return false;
+  for (int ii = max(0, i - l); ii <= min(H - 1, i + l); ++ii)
+    for (int jj = max(0, j - l); jj <= min(W - 1, j + l); ++jj)
+      if ((ii != i || jj != j) && get_bit(rej, Ww, H, b, ii, jj)) return true;
+  return false;
+}
+
+// mulo_resample: one CTA per target position; positions outside R_X copy x~.
+__global__ void __launch_bounds__(kThreads) k_resample_rows(RowKernelArgs a) {
+  __shared__ BlockScratch bs;
+  extern __shared__ __align__(16) unsigned char dyn[];
+  const DevParams& P = a.P;
+  PoolSmem ps = carve_pool(P, dyn);
+  const int N = P.H * P.W, Ww = (P.W + 31) / 32;
+  const size_t g = blockIdx.x;
+  const int b = (int)(g / N), t = (int)(g % N), i = t / P.W, j = t % P.W;
+  const int tok_raw = a.draft_tok_hi[g];
+  if (!get_bit(a.expand_bits, Ww, P.H, b, i, j)) {
+    if (threadIdx.x == 0) a.out_tok[g] = tok_raw;
+    return;
+  }
+  const int rejected = get_bit(a.reject_bits, Ww, P.H, b, i, j);
+  int use_res;
+  if (P.resample_mode == MULO_RESAMPLE_RESIDUAL_ALL) use_res = 1;
+  else if (P.resample_mode == MULO_RESAMPLE_TARGET_ALL) use_res = 0;
+  else if (P.resample_mode == MULO_RESAMPLE_ISOLATED_RESIDUAL) {
+    use_res = rejected;
+    if (rejected) {
+      // first rejection of the image: scan the words of image b (uniform across the CTA)
+      int t0 = N;
+      for (int w = 0; w < P.H * Ww && t0 == N; ++w) {
+        uint32_t v = a.reject_bits[(size_t)b * P.H * Ww + w];
+        if (v) t0 = (w / Ww) * P.W + (w % Ww) * 32 + __ffs(v) - 1;
+      }
+      if (covered_by_other(a.reject_bits, Ww, P.H, P.W, b, i, j, P.radius, P.clip, t0)) use_res = 0;
+    }
+  } else use_res = rejected;
+  const size_t cell = ((size_t)b * P.h + i / P.r) * P.w + j / P.r;
+  RowSrc qr = draft_row(a, cell);
+  RowStats sq;
+  sq.theta = a.stats_in[cell * 4 + 0];
+  sq.m = a.stats_in[cell * 4 + 1];
+  sq.Z = (double)a.stats_in[cell * 4 + 2] + (double)a.stats_in[cell * 4 + 3];
+  const int tok = checked_token(tok_raw, P.V, a.dev_status);
+  RowSrc tr = target_row(a, g);
+  PositionOut o;
+  const int draw = use_res ? kDrawResidual : kDrawTarget;
+  dense_position(P, tr, qr, sq, tok, a.nn, (uint32_t)b + P.image_offset, (uint32_t)t, false, !rejected,
+                 [draw](int) { return draw; }, bs, ps, a.dev_status, o);
+  if (threadIdx.x == 0) a.out_tok[g] = use_res ? o.tok_residual : o.tok_target;
+}
+
+// ============================================================= mask kernel
+// One CTA per image, warps over 32-position tiles: ballot packs accept flags
+// into row words, ffs/popc give t_0 and the counts, funnel shifts dilate.
+
+struct MaskArgs {
+  int H, W, r, radius, clip, resample_mode;
+  const uint8_t* flags;          // [B,H,W] 1 = rejected           (MODE 0, 2)
+  const uint32_t* reject_in;     // [B,H,Ww]                        (MODE 1)
+  const int32_t* first_in;       // [B]                             (MODE 1)
+  uint32_t* reject_bits;         // out (MODE 0, 2)
+  uint32_t* expand_bits;         // out (MODE 1, 2)
+  int32_t* n_reject;             // out (MODE 0, 2), may be null
+  int32_t* first_reject;         // out (MODE 0, 2), may be null
+  int32_t* n_expand;             // out (MODE 1, 2), may be null
+  const int32_t* cand_res;       // MODE 2
+  const int32_t* cand_tgt;       // MODE 2
+  const int32_t* draft_tok_lo;   // MODE 2: [B,h,w]
+  int32_t* out_tok;              // MODE 2
+};
+
+constexpr int kMaskThreads = 256;
+
+// MODE 0: flags -> reject bits, counts, t_0            (tail of mulo_verify)
+// MODE 1: reject bits -> expand bits, count            (mulo_local_reject_expand)
+// MODE 2: flags -> both masks, counts, output tokens   (tail of mulo_round)
+template <int MODE>
+__global__ void __launch_bounds__(kMaskThreads) k_mask(MaskArgs a) {
+  extern __shared__ uint32_t words[];
+  const int H = a.H, W = a.W, Ww = (W + 31) / 32, nw = H * Ww, N = H * W;
+  uint32_t* rej = words;
+  uint32_t* hd = words + nw;
+  uint32_t* ex = words + 2 * nw;
+  __shared__ int s_nrej, s_first, s_nexp;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    s_nrej = 0;
+    s_first = N;
+    s_nexp = 0;
+  }
+  __syncthreads();
+  if (MODE == 1) {
+    for (int w = tid; w < nw; w += kMaskThreads) rej[w] = a.reject_in[(size_t)b * nw + w];
+    if (tid == 0) s_first = a.first_in[b];
+  } else {
+    for (int w = warp; w < nw; w += kMaskThreads / 32) {
+      const int i = w / Ww, j = (w % Ww) * 32 + lane;
+      const bool r = j < W && a.flags[(size_t)b * N + (size_t)i * W + j] != 0;
+      const uint32_t word = __ballot_sync(kFull, r);
+      if (lane == 0) {
+        rej[w] = word;
+        if (word) {
+          atomicAdd(&s_nrej, __popc(word));
+          atomicMin(&s_first, i * W + (w % Ww) * 32 + __ffs(word) - 1);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  const int t0 = s_first;
+  if (MODE != 1) {
+    for (int w = tid; w < nw; w += kMaskThreads) a.reject_bits[(size_t)b * nw + w] = rej[w];
+    if (tid == 0) {
+      if (a.n_reject) a.n_reject[b] = s_nrej;
+      if (a.first_reject) a.first_reject[b] = t0;
+    }
+  }
+  if (MODE == 0) return;
+
+  // horizontal dilation by l: OR of the row shifted by -l..l, with carries
+  // across word boundaries (l <= 31, so only the two adjacent words matter)
+  const int l = a.radius;
+  for (int w = tid; w < nw; w += kMaskThreads) {
+    const int wj = w % Ww;
+    const uint32_t cur = rej[w];
+    const uint32_t prev = wj > 0 ? rej[w - 1] : 0u;
+    const uint32_t next = wj + 1 < Ww ? rej[w + 1] : 0u;
+    uint32_t acc = cur;
+    for (int s = 1; s <= l; ++s) {
+      acc |= __funnelshift_l(prev, cur, s);   // bits moved towards higher j
+      acc |= __funnelshift_r(cur, next, s);   // bits moved towards lower j
+    }
+    if (wj == Ww - 1 && (W & 31)) acc &= (1u << (W & 31)) - 1u;
+    hd[w] = acc;
+  }
+  __syncthreads();
+  // vertical dilation, then Eq. 6's clause u >= t_0
+  for (int w = tid; w < nw; w += kMaskThreads) {
+    const int i = w / Ww, wj = w % Ww;
+    uint32_t acc = 0u;
+    for (int ii = max(0, i - l); ii <= min(H - 1, i + l); ++ii) acc |= hd[ii * Ww + wj];
+    if (a.clip) {
+      const int i0 = t0 / W, j0 = t0 % W;
+      if (t0 >= N || i < i0) acc = (t0 >= N) ? acc : 0u;
+      else if (i == i0) {
+        const int lo = j0 - wj * 32;   // first kept bit of this word
+        if (lo >= 32) acc = 0u;
+        else if (lo > 0) acc &= ~((1u << lo) - 1u);
+      }
+    }
+    ex[w] = acc;
+    a.expand_bits[(size_t)b * nw + w] = acc;
+    if (acc) atomicAdd(&s_nexp, __popc(acc));
+  }
+  __syncthreads();
+  if (tid == 0 && a.n_expand) a.n_expand[b] = s_nexp;
+  if (MODE != 2) return;
+
+  // output assembly: x~ outside R_X, the position's draw inside
+  const int h = H / a.r, w_lo = W / a.r;
+  for (int t = tid; t < N; t += kMaskThreads) {
+    const int i = t / W, j = t % W;
+    const size_t g = (size_t)b * N + t;
+    int tok = a.draft_tok_lo[((size_t)b * h + i / a.r) * w_lo + j / a.r];
+    if ((ex[i * Ww + (j >> 5)] >> (j & 31)) & 1u) {
+      const int rejected = (rej[i * Ww + (j >> 5)] >> (j & 31)) & 1u;
+      int use_res;
+      if (a.resample_mode == MULO_RESAMPLE_RESIDUAL_ALL) use_res = 1;
+      else if (a.resample_mode == MULO_RESAMPLE_TARGET_ALL) use_res = 0;
+      else if (a.resample_mode == MULO_RESAMPLE_ISOLATED_RESIDUAL)
+        use_res = rejected && !covered_by_other(rej, Ww, H, W, 0, i, j, l, a.clip, t0);
+      else use_res = rejected;
+      tok = use_res ? a.cand_res[g] : a.cand_tgt[g];
+    }
+    a.out_tok[g] = tok;
+  }
+}
+
+// ================================================================ host side
+
+struct mulo_ctx {
+  int device;
+  int sm_count;
+  int smem_optin;
+  void* ws;
+  size_t ws_bytes;
+  uint64_t launches;
+};
+
+static const size_t kStatusBytes = 256;
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static mulo_status validate(const mulo_params* p) {
+  if (!p) return MULO_ERR_INVALID_ARG;
+  if (p->B < 0 || p->H <= 0 || p->W <= 0 || p->r <= 0) return MULO_ERR_INVALID_ARG;
+  if (p->H % p->r || p->W % p->r) return MULO_ERR_INVALID_ARG;
+  if (p->V <= 0 || p->V % 8) return MULO_ERR_INVALID_ARG;
+  if (p->logit_dtype != MULO_F32 && p->logit_dtype != MULO_BF16) return MULO_ERR_INVALID_ARG;
+  if (!(p->temperature > 0.0f) || !isfinite(p->temperature)) return MULO_ERR_INVALID_ARG;
+  if (!isfinite(p->cfg_scale)) return MULO_ERR_INVALID_ARG;
+  if (p->accept_mode != MULO_ACCEPT_RATIO && p->accept_mode != MULO_ACCEPT_THRESHOLD) return MULO_ERR_INVALID_ARG;
+  if (p->resample_mode < 0 || p->resample_mode > MULO_RESAMPLE_ISOLATED_RESIDUAL) return MULO_ERR_INVALID_ARG;
+  if (p->radius < 0) return MULO_ERR_INVALID_ARG;
+  if (p->pool_k > 1 && !(p->pool_delta >= 0.0f)) return MULO_ERR_INVALID_ARG;
+  if (p->V > 65536) return MULO_ERR_UNSUPPORTED;
+  if (p->radius > 31) return MULO_ERR_UNSUPPORTED;
+  if (p->pool_k > 2048 || p->pool_k > p->V) return MULO_ERR_UNSUPPORTED;
+  if ((size_t)p->H * ((p->W + 31) / 32) > 4000) return MULO_ERR_UNSUPPORTED;
+  if ((double)p->B * p->H * p->W > 2.0e9) return MULO_ERR_UNSUPPORTED;
+  return MULO_OK;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+static DevParams to_dev(const mulo_params* p) {
+  DevParams d;
+  d.B = p->B; d.H = p->H; d.W = p->W; d.V = p->V; d.r = p->r;
+  d.h = p->H / p->r; d.w = p->W / p->r;
+  d.bf16 = p->logit_dtype == MULO_BF16;
+  d.invT = 1.0f / p->temperature;
+  d.cfg_scale = p->cfg_scale;
+  d.top_k = (p->top_k > 0 && p->top_k < p->V) ? p->top_k : 0;
+  d.accept_mode = p->accept_mode;
+  d.tau = (double)p->tau;
+  d.pool_k = p->pool_k > 1 ? p->pool_k : 1;
+  d.pool_delta = (double)p->pool_delta;
+  d.radius = p->radius; d.clip = p->clip_before_first != 0; d.resample_mode = p->resample_mode;
+  d.seed_lo = (uint32_t)(p->seed & 0xffffffffu); d.seed_hi = (uint32_t)(p->seed >> 32);
+  d.round = p->round; d.image_offset = p->image_offset;
+  return d;
+}
+
+static size_t pool_smem_bytes(const DevParams& d) {
+  if (d.pool_k <= 1) return 0;
+  return (size_t)d.pool_k * sizeof(double) + (size_t)((d.V + 31) / 32) * 4;
+}
+
+struct Workspace {
+  uint32_t* status;
+  uint8_t* flags;
+  int32_t* cand_res;
+  int32_t* cand_tgt;
+  size_t bytes;
+};
+
+static Workspace carve_ws(void* base, const mulo_params* p) {
+  const size_t n = (size_t)p->B * p->H * p->W;
+  Workspace w;
+  char* c = (char*)base;
+  size_t off = 0;
+  w.status = (uint32_t*)(c + off); off += kStatusBytes;
+  w.flags = (uint8_t*)(c + off); off += align_up(n, 256);
+  w.cand_res = (int32_t*)(c + off); off += align_up(n * 4, 256);
+  w.cand_tgt = (int32_t*)(c + off); off += align_up(n * 4, 256);
+  w.bytes = off;
+  return w;
+}
+
+extern "C" {
+
+const char* mulo_status_string(mulo_status s) {
+  switch (s) {
+    case MULO_OK: return "ok";
+    case MULO_ERR_INVALID_ARG: return "invalid argument";
+    case MULO_ERR_UNSUPPORTED: return "unsupported size or parameter";
+    case MULO_ERR_WORKSPACE: return "workspace missing or too small";
+    case MULO_ERR_CUDA: return "CUDA runtime error";
+    case MULO_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+mulo_status mulo_create(mulo_ctx** out, int device) {
+  if (!out) return MULO_ERR_INVALID_ARG;
+  *out = nullptr;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+    cudaGetLastError();
+    return MULO_ERR_CUDA;
+  }
+  if (cudaSetDevice(device) != cudaSuccess) return MULO_ERR_CUDA;
+  mulo_ctx* c = new (std::nothrow) mulo_ctx();
+  if (!c) return MULO_ERR_INVALID_ARG;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  c->smem_optin = (int)prop.sharedMemPerBlockOptin;
+  c->ws = nullptr;
+  c->ws_bytes = 0;
+  c->launches = 0;
+  *out = c;
+  return MULO_OK;
+}
+
+void mulo_destroy(mulo_ctx* ctx) { delete ctx; }
+
+mulo_status mulo_workspace_bytes(const mulo_params* p, size_t* bytes) {
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!bytes) return MULO_ERR_INVALID_ARG;
+  *bytes = carve_ws(nullptr, p).bytes;
+  return MULO_OK;
+}
+
+mulo_status mulo_set_workspace(mulo_ctx* ctx, void* dev_ptr, size_t bytes) {
+  if (!ctx || !dev_ptr || ((uintptr_t)dev_ptr & 255u) || bytes < kStatusBytes) return MULO_ERR_INVALID_ARG;
+  if (cudaMemset(dev_ptr, 0, kStatusBytes) != cudaSuccess) return MULO_ERR_CUDA;
+  ctx->ws = dev_ptr;
+  ctx->ws_bytes = bytes;
+  return MULO_OK;
+}
+
+mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags) {
+  if (!ctx || !flags) return MULO_ERR_INVALID_ARG;
+  if (!ctx->ws) return MULO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(flags, ctx->ws, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MULO_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->ws, 0, sizeof(uint32_t), st) != cudaSuccess) return MULO_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MULO_ERR_CUDA;
+  return MULO_OK;
+}
+
+mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count) {
+  if (!ctx || !count) return MULO_ERR_INVALID_ARG;
+  *count = ctx->launches;
+  return MULO_OK;
+}
+
+}  // extern "C"
+
+static mulo_status check_ws(mulo_ctx* ctx, const mulo_params* p, Workspace* w) {
+  if (!ctx->ws) return MULO_ERR_WORKSPACE;
+  *w = carve_ws(ctx->ws, p);
+  if (w->bytes > ctx->ws_bytes) return MULO_ERR_WORKSPACE;
+  return MULO_OK;
+}
+
+static mulo_status launched(mulo_ctx* ctx, int n) {
+  if (cudaGetLastError() != cudaSuccess) return MULO_ERR_CUDA;
+  ctx->launches += (uint64_t)n;
+  return MULO_OK;
+}
+
+template <class K>
+static bool raise_smem(K kernel, size_t bytes, const mulo_ctx* ctx) {
+  if (bytes + sizeof(BlockScratch) + 1024 > (size_t)ctx->smem_optin) return false;
+  if (bytes > 0)
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+  return true;
+}
+
+static size_t mask_smem(const mulo_params* p) { return (size_t)3 * p->H * ((p->W + 31) / 32) * 4; }
+
+extern "C" {
+
+mulo_status mulo_upsample_pool(mulo_ctx* ctx, const mulo_params* p, const void* draft_logits_lo,
+                               const int32_t* draft_tok_lo, const uint16_t* nn, int32_t* draft_tok_hi,
+                               float* draft_stats_lo, float* q_tok_hi, void* stream) {
+  (void)nn;
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!draft_logits_lo || !draft_tok_lo || !draft_tok_hi || !draft_stats_lo || !q_tok_hi) return MULO_ERR_INVALID_ARG;
+  if (!aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
+  if (!ctx->ws) return MULO_ERR_WORKSPACE;
+  if (p->B == 0) return MULO_OK;
+  RowKernelArgs a;
+  memset(&a, 0, sizeof a);
+  a.P = to_dev(p);
+  a.draft = (const char*)draft_logits_lo;
+  a.draft_tok_lo = draft_tok_lo;
+  a.tok_hi_out = draft_tok_hi;
+  a.stats_out = draft_stats_lo;
+  a.q_tok_hi_out = q_tok_hi;
+  a.dev_status = (uint32_t*)ctx->ws;
+  k_upsample_pool<<<p->B * a.P.h * a.P.w, kThreads, 0, (cudaStream_t)stream>>>(a);
+  return launched(ctx, 1);
+}
+
+mulo_status mulo_verify(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond, const void* tgt_uncond,
+                        const void* draft_logits_lo, const float* draft_stats_lo,
+                        const int32_t* draft_tok_hi, const uint16_t* nn, float* p_tok, float* q_tok,
+                        float* accept_prob, uint32_t* reject_bits, int32_t* n_reject,
+                        int32_t* first_reject, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!tgt_cond || !draft_logits_lo || !draft_stats_lo || !draft_tok_hi || !p_tok || !q_tok || !accept_prob ||
+      !reject_bits || !n_reject || !first_reject)
+    return MULO_ERR_INVALID_ARG;
+  if (p->pool_k > 1 && !nn) return MULO_ERR_INVALID_ARG;
+  if (!aligned16(tgt_cond) || !aligned16(tgt_uncond) || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
+  Workspace w;
+  if ((s = check_ws(ctx, p, &w)) != MULO_OK) return s;
+  if (p->B == 0) return MULO_OK;
+  RowKernelArgs a;
+  memset(&a, 0, sizeof a);
+  a.P = to_dev(p);
+  a.cond = (const char*)tgt_cond;
+  a.uncond = (const char*)tgt_uncond;
+  a.draft = (const char*)draft_logits_lo;
+  a.stats_in = draft_stats_lo;
+  a.draft_tok_hi = draft_tok_hi;
+  a.nn = nn;
+  a.p_tok = p_tok; a.q_tok = q_tok; a.accept_prob = accept_prob;
+  a.flags = w.flags;
+  a.dev_status = w.status;
+  const size_t dyn = pool_smem_bytes(a.P);
+  if (!raise_smem(k_verify_rows<false>, dyn, ctx)) return MULO_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_verify_rows<false><<<(unsigned)((size_t)p->B * p->H * p->W), kThreads, dyn, st>>>(a);
+  MaskArgs m;
+  memset(&m, 0, sizeof m);
+  m.H = p->H; m.W = p->W; m.r = p->r; m.radius = p->radius; m.clip = a.P.clip; m.resample_mode = p->resample_mode;
+  m.flags = w.flags;
+  m.reject_bits = reject_bits; m.n_reject = n_reject; m.first_reject = first_reject;
+  k_mask<0><<<p->B, kMaskThreads, mask_smem(p), st>>>(m);
+  return launched(ctx, 2);
+}
+
+mulo_status mulo_local_reject_expand(mulo_ctx* ctx, const mulo_params* p, const uint32_t* reject_bits,
+                                     const int32_t* first_reject, uint32_t* expand_bits,
+                                     int32_t* n_expand, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!reject_bits || !first_reject || !expand_bits || !n_expand) return MULO_ERR_INVALID_ARG;
+  if (p->B == 0) return MULO_OK;
+  MaskArgs m;
+  memset(&m, 0, sizeof m);
+  m.H = p->H; m.W = p->W; m.r = p->r; m.radius = p->radius; m.clip = p->clip_before_first != 0;
+  m.resample_mode = p->resample_mode;
+  m.reject_in = reject_bits; m.first_in = first_reject;
+  m.expand_bits = expand_bits; m.n_expand = n_expand;
+  k_mask<1><<<p->B, kMaskThreads, mask_smem(p), (cudaStream_t)stream>>>(m);
+  return launched(ctx, 1);
+}
+
+mulo_status mulo_resample(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond, const void* tgt_uncond,
+                          const void* draft_logits_lo, const float* draft_stats_lo,
+                          const int32_t* draft_tok_hi, const uint16_t* nn, const uint32_t* reject_bits,
+                          const uint32_t* expand_bits, int32_t* out_tok, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!tgt_cond || !draft_logits_lo || !draft_stats_lo || !draft_tok_hi || !reject_bits || !expand_bits || !out_tok)
+    return MULO_ERR_INVALID_ARG;
+  if (p->pool_k > 1 && !nn) return MULO_ERR_INVALID_ARG;
+  if (!aligned16(tgt_cond) || !aligned16(tgt_uncond) || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
+  if (!ctx->ws) return MULO_ERR_WORKSPACE;
+  if (p->B == 0) return MULO_OK;
+  RowKernelArgs a;
+  memset(&a, 0, sizeof a);
+  a.P = to_dev(p);
+  a.cond = (const char*)tgt_cond;
+  a.uncond = (const char*)tgt_uncond;
+  a.draft = (const char*)draft_logits_lo;
+  a.stats_in = draft_stats_lo;
+  a.draft_tok_hi = draft_tok_hi;
+  a.nn = nn;
+  a.reject_bits = reject_bits;
+  a.expand_bits = expand_bits;
+  a.out_tok = out_tok;
+  a.dev_status = (uint32_t*)ctx->ws;
+  const size_t dyn = pool_smem_bytes(a.P);
+  if (!raise_smem(k_resample_rows, dyn, ctx)) return MULO_ERR_UNSUPPORTED;
+  k_resample_rows<<<(unsigned)((size_t)p->B * p->H * p->W), kThreads, dyn, (cudaStream_t)stream>>>(a);
+  return launched(ctx, 1);
+}
+
+mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond, const void* tgt_uncond,
+                       const void* draft_logits_lo, const int32_t* draft_tok_lo, const uint16_t* nn,
+                       int32_t* out_tok, uint32_t* reject_bits, uint32_t* expand_bits, float* p_tok,
+                       float* q_tok, float* accept_prob, int32_t* n_reject, int32_t* n_expand,
+                       int32_t* first_reject, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!tgt_cond || !draft_logits_lo || !draft_tok_lo || !out_tok || !reject_bits || !expand_bits)
+    return MULO_ERR_INVALID_ARG;
+  if (p->pool_k > 1 && !nn) return MULO_ERR_INVALID_ARG;
+  if (!aligned16(tgt_cond) || !aligned16(tgt_uncond) || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
+  Workspace w;
+  if ((s = check_ws(ctx, p, &w)) != MULO_OK) return s;
+  if (p->B == 0) return MULO_OK;
+  RowKernelArgs a;
+  memset(&a, 0, sizeof a);
+  a.P = to_dev(p);
+  a.cond = (const char*)tgt_cond;
+  a.uncond = (const char*)tgt_uncond;
+  a.draft = (const char*)draft_logits_lo;
+  a.draft_tok_lo = draft_tok_lo;
+  a.nn = nn;
+  a.p_tok = p_tok; a.q_tok = q_tok; a.accept_prob = accept_prob;
+  a.flags = w.flags; a.cand_res = w.cand_res; a.cand_tgt = w.cand_tgt;
+  a.dev_status = w.status;
+  const size_t dyn = pool_smem_bytes(a.P);
+  if (!raise_smem(k_verify_rows<true>, dyn, ctx)) return MULO_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_verify_rows<true><<<p->B * a.P.h * a.P.w, kThreads, dyn, st>>>(a);
+  MaskArgs m;
+  memset(&m, 0, sizeof m);
+  m.H = p->H; m.W = p->W; m.r = p->r; m.radius = p->radius; m.clip = a.P.clip; m.resample_mode = p->resample_mode;
+  m.flags = w.flags;
+  m.reject_bits = reject_bits; m.expand_bits = expand_bits;
+  m.n_reject = n_reject; m.first_reject = first_reject; m.n_expand = n_expand;
+  m.cand_res = w.cand_res; m.cand_tgt = w.cand_tgt;
+  m.draft_tok_lo = draft_tok_lo; m.out_tok = out_tok;
+  k_mask<2><<<p->B, kMaskThreads, mask_smem(p), st>>>(m);
+  return launched(ctx, 2);
+}
+
+// ---- host-buffer variant -------------------------------------------------------------
+
+struct HostArena {
+  size_t ws, cond, uncond, draft, tok_lo, nn, out_tok, rbits, ebits, ptok, qtok, aprob, nrej, nexp, first, total;
+};
+
+static HostArena carve_arena(const mulo_params* p, int has_uncond) {
+  const size_t n = (size_t)p->B * p->H * p->W, nlo = n / ((size_t)p->r * p->r);
+  const size_t esz = p->logit_dtype == MULO_BF16 ? 2 : 4;
+  const size_t nwords = (size_t)p->B * p->H * ((p->W + 31) / 32);
+  HostArena a;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes ? bytes : 1, 256); return o; };
+  a.ws = take(carve_ws(nullptr, p).bytes);
+  a.cond = take(n * p->V * esz);
+  a.uncond = take(has_uncond ? n * p->V * esz : 0);
+  a.draft = take(nlo * p->V * esz);
+  a.tok_lo = take(nlo * 4);
+  a.nn = take(p->pool_k > 1 ? (size_t)p->V * p->pool_k * 2 : 0);
+  a.out_tok = take(n * 4);
+  a.rbits = take(nwords * 4);
+  a.ebits = take(nwords * 4);
+  a.ptok = take(n * 4); a.qtok = take(n * 4); a.aprob = take(n * 4);
+  a.nrej = take((size_t)p->B * 4); a.nexp = take((size_t)p->B * 4); a.first = take((size_t)p->B * 4);
+  a.total = off;
+  return a;
+}
+
+mulo_status mulo_round_host_arena_bytes(const mulo_params* p, int has_uncond, size_t* bytes) {
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!bytes) return MULO_ERR_INVALID_ARG;
+  *bytes = carve_arena(p, has_uncond).total;
+  return MULO_OK;
+}
+
+mulo_status mulo_round_host(mulo_ctx* ctx, const mulo_params* p, void* arena, size_t arena_bytes,
+                            const void* tgt_cond, const void* tgt_uncond, const void* draft_logits_lo,
+                            const int32_t* draft_tok_lo, const uint16_t* nn, int32_t* out_tok,
+                            uint32_t* reject_bits, uint32_t* expand_bits, float* p_tok, float* q_tok,
+                            float* accept_prob, int32_t* n_reject, int32_t* n_expand,
+                            int32_t* first_reject, void* stream) {
+  if (!ctx || !arena || ((uintptr_t)arena & 255u)) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!tgt_cond || !draft_logits_lo || !draft_tok_lo || !out_tok || !reject_bits || !expand_bits)
+    return MULO_ERR_INVALID_ARG;
+  if (p->pool_k > 1 && !nn) return MULO_ERR_INVALID_ARG;
+  const HostArena A = carve_arena(p, tgt_uncond != nullptr);
+  if (A.total > arena_bytes) return MULO_ERR_WORKSPACE;
+  if (p->B == 0) return MULO_OK;
+  char* d = (char*)arena;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t n = (size_t)p->B * p->H * p->W, nlo = n / ((size_t)p->r * p->r);
+  const size_t esz = p->logit_dtype == MULO_BF16 ? 2 : 4;
+  const size_t nwords = (size_t)p->B * p->H * ((p->W + 31) / 32);
+  bool ok = true;
+  ok &= cudaMemsetAsync(d + A.ws, 0, kStatusBytes, st) == cudaSuccess;
+  ctx->ws = d + A.ws;
+  ctx->ws_bytes = carve_ws(nullptr, p).bytes;
+  ok &= cudaMemcpyAsync(d + A.draft, draft_logits_lo, nlo * p->V * esz, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d + A.tok_lo, draft_tok_lo, nlo * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (p->pool_k > 1)
+    ok &= cudaMemcpyAsync(d + A.nn, nn, (size_t)p->V * p->pool_k * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d + A.cond, tgt_cond, n * p->V * esz, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (tgt_uncond)
+    ok &= cudaMemcpyAsync(d + A.uncond, tgt_uncond, n * p->V * esz, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) return MULO_ERR_CUDA;
+  s = mulo_round(ctx, p, d + A.cond, tgt_uncond ? d + A.uncond : nullptr, d + A.draft,
+                 (const int32_t*)(d + A.tok_lo), p->pool_k > 1 ? (const uint16_t*)(d + A.nn) : nullptr,
+                 (int32_t*)(d + A.out_tok), (uint32_t*)(d + A.rbits), (uint32_t*)(d + A.ebits),
+                 p_tok ? (float*)(d + A.ptok) : nullptr, q_tok ? (float*)(d + A.qtok) : nullptr,
+                 accept_prob ? (float*)(d + A.aprob) : nullptr, (int32_t*)(d + A.nrej),
+                 (int32_t*)(d + A.nexp), (int32_t*)(d + A.first), stream);
+  if (s != MULO_OK) return s;
+  ok &= cudaMemcpyAsync(out_tok, d + A.out_tok, n * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(reject_bits, d + A.rbits, nwords * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(expand_bits, d + A.ebits, nwords * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (p_tok) ok &= cudaMemcpyAsync(p_tok, d + A.ptok, n * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (q_tok) ok &= cudaMemcpyAsync(q_tok, d + A.qtok, n * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (accept_prob) ok &= cudaMemcpyAsync(accept_prob, d + A.aprob, n * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (n_reject) ok &= cudaMemcpyAsync(n_reject, d + A.nrej, (size_t)p->B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (n_expand) ok &= cudaMemcpyAsync(n_expand, d + A.nexp, (size_t)p->B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (first_reject) ok &= cudaMemcpyAsync(first_reject, d + A.first, (size_t)p->B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? MULO_OK : MULO_ERR_CUDA;
+}
+
+}  // extern "C"

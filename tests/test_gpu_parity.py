@@ -1,0 +1,218 @@
+"""GPU parity: the CUDA round, called through the C ABI, against the CPU oracle
+on the same seeded inputs -- decisions, masks and tokens bit for bit (borderline
+uniforms excepted and counted), probabilities within the stated tolerances."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_05149_b200 import binding, synth
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    assert torch.cuda.is_available()
+    binding.lib()            # raises if the library was not built: no fallback
+    c = binding.Context(0)
+    yield c
+    assert c.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
+    c.close()
+
+
+TINY = synth.RoundConfig("tiny", B=2, H=8, W=8, V=256, dtype="f32", sigma=1.0, radius=1, seed=101)
+
+
+def _run(ctx, cfg, images=None, **over):
+    batch = pu.build_batch(cfg)
+    g = pu.gpu_round(ctx, cfg, batch, **over)
+    images = list(range(cfg.B)) if images is None else images
+    o = pu.oracle_images(cfg, batch, images, **over)
+    return batch, g, o
+
+
+@pytest.mark.parametrize("cfg", [
+    TINY,
+    dataclasses.replace(TINY, dtype="bf16", seed=102),
+    dataclasses.replace(TINY, dtype="bf16", top_k=40, seed=103),
+    dataclasses.replace(TINY, dtype="f32", top_k=40, cfg_scale=3.0, temperature=0.7, seed=104),
+    dataclasses.replace(TINY, dtype="bf16", top_k=40, cfg_scale=3.0, radius=2, seed=105),
+    dataclasses.replace(TINY, V=264, H=6, W=10, r=1, top_k=17, seed=106),          # ragged sizes
+    dataclasses.replace(TINY, V=8, H=4, W=4, top_k=3, seed=107),                    # tiny vocabulary
+    dataclasses.replace(TINY, H=12, W=36, r=3, radius=3, dtype="bf16", seed=108),   # two mask words per row
+    dataclasses.replace(TINY, V=2048, top_k=300, pool_k=128, pool_delta=0.1, dtype="bf16", seed=109),
+    dataclasses.replace(TINY, V=2048, top_k=0, pool_k=64, pool_delta=0.3, dtype="f32", seed=110),
+], ids=lambda c: f"{c.dtype}-V{c.V}-k{c.top_k}-cfg{c.cfg_scale}-pool{c.pool_k}-{c.H}x{c.W}r{c.r}l{c.radius}")
+def test_round_small(ctx, cfg):
+    batch, g, o = _run(ctx, cfg)
+    pu.check_round(cfg, g, o)
+    # something was rejected and something was swept in, or the case tests nothing
+    assert g["n_reject"].sum() > 0 and g["n_expand"].sum() > g["n_reject"].sum()
+
+
+@pytest.mark.parametrize("mode", [binding.RESAMPLE_MIXED, binding.RESAMPLE_RESIDUAL_ALL,
+                                  binding.RESAMPLE_TARGET_ALL, binding.RESAMPLE_ISOLATED_RESIDUAL])
+@pytest.mark.parametrize("clip", [0, 1])
+def test_round_modes(ctx, mode, clip):
+    cfg = dataclasses.replace(TINY, dtype="bf16", top_k=60, radius=2, seed=120 + mode,
+                              resample_mode=mode, clip_before_first=clip)
+    batch, g, o = _run(ctx, cfg)
+    pu.check_round(cfg, g, o)
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-3, 1e-4, 1.5])
+def test_round_threshold_rule(ctx, tau):
+    """The relaxed rule of Eq. 5 with redraws from the target distribution."""
+    cfg = dataclasses.replace(TINY, dtype="bf16", V=2048, top_k=300, pool_k=64, pool_delta=0.1, seed=130,
+                              accept_mode=binding.ACCEPT_THRESHOLD, tau=tau,
+                              resample_mode=binding.RESAMPLE_TARGET_ALL)
+    batch, g, o = _run(ctx, cfg)
+    pu.check_round(cfg, g, o)
+    if tau == 0.0:
+        assert g["n_reject"].sum() == 0
+    if tau > 1:
+        assert g["reject"].all() and g["expand"].all()
+
+
+def test_identity_target_equals_draft(ctx):
+    cfg = dataclasses.replace(TINY, dtype="bf16", top_k=40, sigma=0.0, seed=140)
+    batch, g, o = _run(ctx, cfg)
+    assert g["n_reject"].sum() == 0 and g["n_expand"].sum() == 0
+    assert np.all(g["accept_prob"] == 1.0)
+    assert np.array_equal(g["out_tok"], batch["tok_lo"].cpu().numpy().repeat(2, 1).repeat(2, 2))
+    assert np.all(g["first_reject"] == cfg.H * cfg.W)
+    pu.check_round(cfg, g, o)
+
+
+def test_stages_equal_fused(ctx):
+    """upsample_pool -> verify -> local_reject_expand -> resample gives exactly
+    the fused round; each stage is also checked against the oracle."""
+    import oracle as orc
+    for cfg in (dataclasses.replace(TINY, dtype="bf16", top_k=40, cfg_scale=3.0, radius=2, seed=150),
+                dataclasses.replace(TINY, V=2048, top_k=300, pool_k=128, dtype="bf16", seed=151,
+                                    resample_mode=binding.RESAMPLE_ISOLATED_RESIDUAL)):
+        batch = pu.build_batch(cfg)
+        f = pu.gpu_round(ctx, cfg, batch)
+        s = pu.gpu_stages(ctx, cfg, batch)
+        for k in ("out_tok", "reject_bits", "expand_bits", "n_reject", "n_expand", "first_reject",
+                  "p_tok", "q_tok", "accept_prob"):
+            assert np.array_equal(f[k], s[k]), k
+        o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
+        pu.check_round(cfg, s, o)
+        for b in range(cfg.B):
+            up = orc.upsample_pool_image(pu.orc_params(cfg, b), synth.to_numpy_logits(batch["draft_lo"][b]),
+                                         batch["tok_lo"][b].cpu().numpy())
+            assert np.array_equal(s["tok_hi"][b], up["tok_hi"])
+            assert np.array_equal(s["stats"][b][..., 0], up["stats"][..., 0].astype(np.float32))
+            assert np.array_equal(s["stats"][b][..., 1], up["stats"][..., 1].astype(np.float32))
+            Zq = s["stats"][b][..., 2].astype(np.float64) + s["stats"][b][..., 3]
+            assert np.allclose(Zq, up["stats"][..., 2], rtol=1e-7)
+            assert np.allclose(s["q_tok_hi"][b], up["q_tok"], rtol=2e-6)
+            assert np.array_equal(s["q_tok_hi"][b], s["q_tok"][b])
+
+
+def test_expand_stage_against_oracle(ctx):
+    """mulo_local_reject_expand alone on random masks, all radii, clip on/off."""
+    import oracle as orc
+    rng = np.random.default_rng(7)
+    for (H, W) in ((5, 7), (16, 16), (9, 70), (64, 64)):
+        for l in (0, 1, 2, 3, 5, 9):
+            for clip in (0, 1):
+                B = 3
+                rej = (rng.random((B, H, W)) < rng.choice([0.0, 0.01, 0.1])).astype(np.uint8)
+                Ww = (W + 31) // 32
+                padded = np.zeros((B, H, Ww * 32), np.uint8)
+                padded[..., :W] = rej
+                words = (padded.reshape(B, H, Ww, 32).astype(np.uint64) << np.arange(32, dtype=np.uint64)).sum(-1)
+                words = words.astype(np.uint32)
+                first = np.array([np.flatnonzero(r.ravel())[0] if r.any() else H * W for r in rej], np.int32)
+                p = binding.make_params(B, H, W, 8, 1, binding.F32, radius=l, clip_before_first=clip)
+                d_rej = torch.from_numpy(words.view(np.int32)).cuda()
+                d_first = torch.from_numpy(first).cuda()
+                d_exp = torch.empty_like(d_rej)
+                d_n = torch.empty(B, dtype=torch.int32, device="cuda")
+                ctx.mulo_local_reject_expand(p, d_rej, d_first, d_exp, d_n)
+                got = binding.unpack_bits(d_exp, W).numpy()
+                for b in range(B):
+                    want, t0 = orc.expand(rej[b], l, clip)
+                    assert np.array_equal(got[b], want), (H, W, l, clip, b)
+                    assert int(d_n[b]) == want.sum()
+
+
+def test_config_C1(ctx):
+    cfg = synth.CONFIGS["C1"]
+    batch, g, o = _run(ctx, cfg)
+    pu.check_round(cfg, g, o)
+
+
+def test_config_C2(ctx):
+    cfg = synth.CONFIGS["C2"]
+    batch = pu.build_batch(cfg)
+    g = pu.gpu_round(ctx, cfg, batch)
+    o = pu.oracle_images(cfg, batch, [0])
+    pu.check_round(cfg, g, o)
+
+
+def test_config_C3_sampled_images(ctx):
+    """Full-size batch on the GPU, first and last image against the oracle."""
+    cfg = synth.CONFIGS["C3"]
+    batch = pu.build_batch(cfg)
+    g = pu.gpu_round(ctx, cfg, batch)
+    o = pu.oracle_images(cfg, batch, [0, cfg.B - 1])
+    pu.check_round(cfg, g, o)
+
+
+def test_rounds_and_image_offset_change_the_draws(ctx):
+    cfg = dataclasses.replace(TINY, dtype="bf16", top_k=40, seed=160)
+    batch = pu.build_batch(cfg)
+    a = pu.gpu_round(ctx, cfg, batch)
+    b = pu.gpu_round(ctx, cfg, batch, round=1)
+    assert not np.array_equal(a["reject"], b["reject"])
+    # image_offset shifts the Philox image index: image 0 with offset 1 uses image 1's stream
+    c = pu.gpu_round(ctx, cfg, batch, image_offset=5)
+    o = pu.oracle_images(cfg, batch, [0, 1], image_offset=5)
+    pu.check_round(cfg, c, o)
+    # a repeated call is bit-identical
+    a2 = pu.gpu_round(ctx, cfg, batch)
+    for k in a:
+        assert np.array_equal(a[k], a2[k])
+
+
+def test_host_buffer_round(ctx):
+    cfg = dataclasses.replace(TINY, dtype="bf16", top_k=40, cfg_scale=3.0, seed=170)
+    batch = pu.build_batch(cfg)
+    ref = pu.gpu_round(ctx, cfg, batch)
+    p = binding.params_from_config(cfg)
+    arena = torch.empty(binding.Context.round_host_arena_bytes(p, True), dtype=torch.uint8, device="cuda")
+    host = {k: (None if v is None else v.cpu().pin_memory()) for k, v in batch.items()}
+    o = binding.alloc_round_outputs(p, "cpu", True)
+    c2 = binding.Context(0)
+    c2.mulo_round_host(p, arena, host["cond"], host["uncond"], host["draft_lo"], host["tok_lo"], host["nn"],
+                       o["out_tok"], o["reject_bits"], o["expand_bits"], o["p_tok"], o["q_tok"],
+                       o["accept_prob"], o["n_reject"], o["n_expand"], o["first_reject"])
+    for k in ("out_tok", "reject_bits", "expand_bits", "p_tok", "q_tok", "accept_prob", "n_reject",
+              "n_expand", "first_reject"):
+        assert np.array_equal(o[k].numpy(), ref[k]), k
+    c2.close()
+
+
+def test_device_status_reports_contract_violations(ctx):
+    cfg = dataclasses.replace(TINY, dtype="bf16", top_k=4, seed=180)
+    batch = pu.build_batch(cfg)
+    assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
+    bad = dict(batch)
+    bad["tok_lo"] = batch["tok_lo"].clone()
+    bad["tok_lo"][0, 0, 0] = cfg.V + 5                 # outside the vocabulary
+    pu.gpu_round(ctx, cfg, bad)
+    assert ctx.poll_device_status() & binding.DEV_BAD_TOKEN
+    # a token outside the draft top-k has q = 0
+    worst = batch["draft_lo"][0, 0, 0].float().argmin().item()
+    bad["tok_lo"] = batch["tok_lo"].clone()
+    bad["tok_lo"][0, 0, 0] = worst
+    pu.gpu_round(ctx, cfg, bad)
+    assert ctx.poll_device_status() & binding.DEV_ZERO_DRAFT_PROB
+    assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0      # reading clears
