@@ -1,0 +1,341 @@
+"""Benchmark of the fused MuLo-SD draft-and-verify round.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C4] [--impl ours|reference]
+
+A step is one fused round (``mulo_round``) over one batch of synthetic logits that
+is already resident in HBM.  Prints ONE JSON line: verified grid positions per
+second (whole job), the HBM roofline of the row kernel, the same metric end to end
+from host buffers, and the CPU oracle timed on a bounded sample of the workload.
+Under torchrun (N > 1) every rank runs the same batch shape on its own GPU
+(independent images, no collective on the data path; image_offset = rank * B).
+"""
+from __future__ import annotations
+
+import argparse
+import concurrent.futures as cf
+import dataclasses
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2601_05149_b200 import synth  # noqa: E402
+
+METRIC = "verified_grid_positions_per_sec"
+UNIT = "positions/s"
+
+
+def workload_desc(cfg):
+    return (f"{cfg.name}: B={cfg.B} target {cfg.H}x{cfg.W} / draft {cfg.h}x{cfg.w}, V={cfg.V}, {cfg.dtype} "
+            f"logits, CFG {cfg.cfg_scale}, top-k {cfg.top_k}, pool_k {cfg.pool_k}, radius {cfg.radius}, "
+            f"sigma {cfg.sigma}")
+
+
+# ----------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------- CPU oracle
+
+def _crop_for_oracle(cfg, rows=16):
+    """A bounded sample of the workload for the CPU oracle: the first `rows` grid rows
+    of an image (same V, dtype, knobs), one such crop per host thread."""
+    rows = min(rows, cfg.H)
+    rows -= rows % cfg.r
+    return dataclasses.replace(cfg, name=cfg.name + "-crop", B=1, H=rows)
+
+
+def time_oracle(cfg, steps, warmup, cores=None):
+    """Times the oracle as it stands on this host: `cores` threads, each running the
+    whole round on its own crop.  Returns (positions/s, per-step seconds, cores, sample)."""
+    import oracle as orc
+    cores = cores or min(os.cpu_count() or 1, 16)
+    crop = _crop_for_oracle(cfg)
+    inputs = []
+    for b in range(cores):
+        img = synth.make_image(dataclasses.replace(cfg, H=cfg.H), b, "cpu")
+        tok = synth.draw_draft_tokens(cfg, b, img["draft_lo"])
+        cut = lambda t, n: None if t is None else synth.to_numpy_logits(t[:n].contiguous())
+        inputs.append((cut(img["cond"], crop.H), cut(img["uncond"], crop.H), cut(img["draft_lo"], crop.h),
+                       tok[:crop.h].contiguous().numpy()))
+    nn = None
+    if cfg.pool_k > 1:
+        nn = synth.neighbours_to_numpy(synth.codebook_neighbours(cfg.V, cfg.pool_k, cfg.seed))
+    orc.lib()
+
+    def one(args):
+        b, rnd = args
+        c, u, d, t = inputs[b]
+        prm = orc.make_params(
+            crop.H, crop.W, crop.V, crop.r, orc.BF16 if crop.dtype == "bf16" else orc.F32,
+            temperature=crop.temperature, top_k=crop.top_k, cfg_scale=crop.cfg_scale,
+            accept_mode=crop.accept_mode, tau=crop.tau, pool_k=crop.pool_k, pool_delta=crop.pool_delta,
+            radius=crop.radius, clip_before_first=crop.clip_before_first, resample_mode=crop.resample_mode,
+            seed=crop.seed, round=rnd, image=b)
+        return orc.round_image(prm, c, u, d, t, nn)
+
+    times = []
+    with cf.ThreadPoolExecutor(max_workers=cores) as ex:
+        for s in range(warmup + steps):
+            t0 = time.perf_counter()
+            list(ex.map(one, [(b, s) for b in range(cores)]))
+            dt = time.perf_counter() - t0
+            if s >= warmup:
+                times.append(dt)
+    per_step = sum(times) / len(times)
+    positions = cores * crop.H * crop.W
+    sample = (f"{cores} threads x one {crop.H}x{crop.W} crop (first {crop.H} grid rows) of a {cfg.name} image, "
+              f"{positions} positions per step")
+    return positions / per_step, per_step, cores, sample
+
+
+# ------------------------------------------------------------------- arms
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, args.steps)
+    warmup = max(0, min(args.warmup, 2))
+    value, per_step, cores, sample = time_oracle(cfg, steps, warmup)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_desc(cfg), "note": "CPU oracle on a bounded sample of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours(args, cfg):
+    from paper_2601_05149_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the round has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.lib()
+    ctx = binding.Context(local)
+    dev = torch.device("cuda", local)
+
+    # this rank's images: global indices [rank*B, (rank+1)*B)
+    rcfg = dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+    batch = synth.build_batch(rcfg, dev)
+    p = binding.params_from_config(cfg, image_offset=rank * cfg.B)
+    ctx.ensure_workspace(p)
+    out = binding.alloc_round_outputs(p, dev, probs=False)
+    stream = torch.cuda.current_stream()
+
+    def step(rnd):
+        p.round = rnd
+        ctx.mulo_round(p, batch["cond"], batch["uncond"], batch["draft_lo"], batch["tok_lo"], batch["nn"],
+                       out["out_tok"], out["reject_bits"], out["expand_bits"], None, None, None,
+                       out["n_reject"], out["n_expand"], out["first_reject"], stream)
+
+    W, K = max(3, args.warmup), max(1, args.steps)
+    for s in range(W):
+        step(s)
+    torch.cuda.synchronize()
+    ctx.set_timing(K)
+    launches0 = ctx.kernel_launches()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record(stream)
+    for s in range(K):
+        step(W + s)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    elapsed_ms = e0.elapsed_time(e1)
+    row_ms, row_n = ctx.read_timing()
+    ctx.set_timing(0)
+    launches = ctx.kernel_launches() - launches0
+    if dist:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    positions = cfg.B * cfg.H * cfg.W
+    value = world * positions * K / (elapsed_ms * 1e-3)
+    n_rej = int(out["n_reject"].sum().item())
+    n_exp = int(out["n_expand"].sum().item())
+    status = ctx.poll_device_status()
+
+    # roofline of the row kernel: algorithmic bytes of one launch / its mean duration
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = 6650.0, "fallback (6.65 TB/s)"
+    alg_bytes = cfg.algorithmic_bytes_per_position() * positions
+    row_avg_ms = row_ms / max(1, row_n)
+    achieved = alg_bytes / (row_avg_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "k_verify_rows<fused>", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                "frac_of_nominal_8TBps": achieved / 8000.0, "traffic": None,
+                "bytes_per_launch": alg_bytes, "avg_launch_ms": row_avg_ms, "launches_timed": row_n}
+    tr = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tr):
+        try:
+            roofline["traffic"] = json.load(open(tr)).get(cfg.name)
+        except (ValueError, OSError):
+            pass
+
+    e2e = None
+    cpu = None
+    if rank == 0:
+        e2e = run_e2e(ctx, cfg, p, batch, world, args)
+    if dist:
+        dist.barrier()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, per_step, cores, sample = time_oracle(cfg, steps=1, warmup=0)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+               "seconds": per_step}
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_desc(cfg), "per_gpu_batch": cfg.B,
+                       "l2": "inputs per step (%.2f GB) exceed the 126 MB L2; no flush needed" % (alg_bytes / 1e9),
+                       "acceptance_rate": 1.0 - n_rej / positions, "expanded_fraction": n_exp / positions,
+                       "device_status": status},
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        }))
+    ctx.close()
+    if dist:
+        dist.destroy_process_group()
+
+
+def run_e2e(ctx, cfg, p, batch, world, args):
+    """The same round through mulo_round_host: pinned host inputs copied to the device,
+    results copied back, all inside the timed region (rank 0's GPU; at N > 1 the other
+    ranks idle, so this is a single-GPU figure scaled by nothing)."""
+    from paper_2601_05149_b200 import binding
+    dev = batch["cond"].device
+    try:
+        host = {k: (None if v is None else v.cpu().pin_memory()) for k, v in batch.items()}
+    except RuntimeError as e:
+        return {"value": None, "unit": UNIT, "error": f"pinning host memory failed: {e}"}
+    arena = torch.empty(binding.Context.round_host_arena_bytes(p, cfg.has_uncond), dtype=torch.uint8, device=dev)
+    o = binding.alloc_round_outputs(p, "cpu", probs=False)
+    o = {k: v.pin_memory() for k, v in o.items()}
+    c2 = binding.Context(dev.index)
+    stream = torch.cuda.current_stream()
+    steps = max(1, min(args.steps, 3))
+
+    def step(rnd):
+        p.round = rnd
+        c2.mulo_round_host(p, arena, host["cond"], host["uncond"], host["draft_lo"], host["tok_lo"], host["nn"],
+                           o["out_tok"], o["reject_bits"], o["expand_bits"], None, None, None,
+                           o["n_reject"], o["n_expand"], o["first_reject"], stream)
+
+    step(0)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(steps):
+        step(1 + s)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    h2d = sum(v.numel() * v.element_size() for v in host.values() if v is not None)
+    d2h = sum(v.numel() * v.element_size() for v in o.values())
+    c2.close()
+    return {"value": cfg.B * cfg.H * cfg.W / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "n_gpus": 1}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C4", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = synth.CONFIGS[args.workload]
+    if args.batch:
+        cfg = dataclasses.replace(cfg, B=args.batch, name=f"{cfg.name}(B={args.batch})")
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -121,6 +121,13 @@ mulo_status mulo_set_workspace(mulo_ctx* ctx, void* dev_ptr, size_t bytes);
 mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags);
 /* Number of kernels this context has launched so far. */
 mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
+/* Optional device timing of the fused row kernel (the launch that reads the logits):
+ * mulo_set_timing prepares CUDA event pairs for up to max_launches (<= 4096) calls of
+ * mulo_round (0 turns timing off); every mulo_round then records an event on its stream
+ * before and after that kernel.  mulo_read_timing waits for the recorded launches, returns
+ * their summed duration in milliseconds and their number, and starts a new series. */
+mulo_status mulo_set_timing(mulo_ctx* ctx, int max_launches);
+mulo_status mulo_read_timing(mulo_ctx* ctx, double* row_kernel_ms, uint64_t* row_kernel_launches);
 
 /* ---- the four stages ------------------------------------------------------------------ */
 

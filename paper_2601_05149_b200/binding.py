@@ -23,6 +23,7 @@ DEV_ZERO_DRAFT_PROB, DEV_BAD_TOKEN, DEV_DENSE_FALLBACK = 1, 2, 4
 EXPORTS = (
     "mulo_create", "mulo_destroy", "mulo_status_string", "mulo_workspace_bytes",
     "mulo_set_workspace", "mulo_poll_device_status", "mulo_kernel_launches",
+    "mulo_set_timing", "mulo_read_timing",
     "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_resample",
     "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host",
 )
@@ -176,6 +177,15 @@ class Context:
         n = C.c_uint64()
         _check(lib().mulo_kernel_launches(self._ctx, C.byref(n)), "mulo_kernel_launches")
         return n.value
+
+    def set_timing(self, max_launches: int):
+        _check(lib().mulo_set_timing(self._ctx, int(max_launches)), "mulo_set_timing")
+
+    def read_timing(self):
+        """(summed milliseconds, launches) of the fused row kernel since the last read."""
+        ms, n = C.c_double(), C.c_uint64()
+        _check(lib().mulo_read_timing(self._ctx, C.byref(ms), C.byref(n)), "mulo_read_timing")
+        return ms.value, n.value
 
     # -- stages ------------------------------------------------------------
     def mulo_upsample_pool(self, p, draft_logits_lo, draft_tok_lo, nn, draft_tok_hi, draft_stats_lo,

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "../../include/mulo.h"
 #include "mulo_dense.cuh"
@@ -373,6 +374,8 @@ struct mulo_ctx {
   void* ws;
   size_t ws_bytes;
   uint64_t launches;
+  std::vector<cudaEvent_t> ev;   // start/stop pairs around the fused row kernel
+  size_t ev_used;
 };
 
 static const size_t kStatusBytes = 256;
@@ -476,11 +479,44 @@ mulo_status mulo_create(mulo_ctx** out, int device) {
   c->ws = nullptr;
   c->ws_bytes = 0;
   c->launches = 0;
+  c->ev_used = 0;
   *out = c;
   return MULO_OK;
 }
 
-void mulo_destroy(mulo_ctx* ctx) { delete ctx; }
+void mulo_destroy(mulo_ctx* ctx) {
+  if (!ctx) return;
+  for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+  delete ctx;
+}
+
+mulo_status mulo_set_timing(mulo_ctx* ctx, int max_launches) {
+  if (!ctx || max_launches < 0 || max_launches > 4096) return MULO_ERR_INVALID_ARG;
+  for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+  ctx->ev.clear();
+  ctx->ev_used = 0;
+  for (int i = 0; i < 2 * max_launches; ++i) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return MULO_ERR_CUDA;
+    ctx->ev.push_back(e);
+  }
+  return MULO_OK;
+}
+
+mulo_status mulo_read_timing(mulo_ctx* ctx, double* row_kernel_ms, uint64_t* row_kernel_launches) {
+  if (!ctx || !row_kernel_ms || !row_kernel_launches) return MULO_ERR_INVALID_ARG;
+  double total = 0.0;
+  for (size_t i = 0; i + 1 < ctx->ev_used; i += 2) {
+    if (cudaEventSynchronize(ctx->ev[i + 1]) != cudaSuccess) return MULO_ERR_CUDA;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->ev[i], ctx->ev[i + 1]) != cudaSuccess) return MULO_ERR_CUDA;
+    total += ms;
+  }
+  *row_kernel_ms = total;
+  *row_kernel_launches = ctx->ev_used / 2;
+  ctx->ev_used = 0;
+  return MULO_OK;
+}
 
 mulo_status mulo_workspace_bytes(const mulo_params* p, size_t* bytes) {
   mulo_status s = validate(p);
@@ -688,7 +724,13 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   const size_t dyn = pool_smem_bytes(a.P);
   if (!raise_smem(k_verify_rows<true>, dyn, ctx)) return MULO_ERR_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
+  const bool timed = ctx->ev_used + 2 <= ctx->ev.size();
+  if (timed) cudaEventRecord(ctx->ev[ctx->ev_used], st);
   k_verify_rows<true><<<p->B * a.P.h * a.P.w, kThreads, dyn, st>>>(a);
+  if (timed) {
+    cudaEventRecord(ctx->ev[ctx->ev_used + 1], st);
+    ctx->ev_used += 2;
+  }
   MaskArgs m;
   memset(&m, 0, sizeof m);
   m.H = p->H; m.W = p->W; m.r = p->r; m.radius = p->radius; m.clip = a.P.clip; m.resample_mode = p->resample_mode;

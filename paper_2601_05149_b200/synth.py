@@ -175,3 +175,26 @@ def to_numpy_logits(t: torch.Tensor) -> np.ndarray:
 
 def neighbours_to_numpy(nn: torch.Tensor) -> np.ndarray:
     return nn.detach().cpu().numpy().astype(np.uint16)
+
+
+def build_batch(cfg: RoundConfig, device="cuda"):
+    """All inputs of one round as device tensors."""
+    dt = cfg.torch_dtype
+    cond = torch.empty((cfg.B, cfg.H, cfg.W, cfg.V), dtype=dt, device=device)
+    uncond = torch.empty_like(cond) if cfg.has_uncond else None
+    draft = torch.empty((cfg.B, cfg.h, cfg.w, cfg.V), dtype=dt, device=device)
+    tok = torch.empty((cfg.B, cfg.h, cfg.w), dtype=torch.int32, device=device)
+    for b in range(cfg.B):
+        img = make_image(cfg, b, device)
+        cond[b] = img["cond"]
+        if uncond is not None:
+            uncond[b] = img["uncond"]
+        draft[b] = img["draft_lo"]
+        tok[b] = draw_draft_tokens(cfg, b, img["draft_lo"])
+        del img
+    nn = None
+    if cfg.pool_k > 1:
+        # uint16 ids, carried in an int16 tensor (same bit pattern)
+        ids = neighbours_to_numpy(codebook_neighbours(cfg.V, cfg.pool_k, cfg.seed, device))
+        nn = torch.from_numpy(ids.view(np.int16)).to(device).contiguous()
+    return dict(cond=cond, uncond=uncond, draft_lo=draft, tok_lo=tok, nn=nn)
