@@ -76,6 +76,7 @@ typedef enum {
 #define MULO_DEV_ZERO_DRAFT_PROB 1u /* some draft token had q(x~) == 0                    */
 #define MULO_DEV_BAD_TOKEN 2u       /* some token / neighbour id was outside [0, V)        */
 #define MULO_DEV_DENSE_FALLBACK 4u  /* informational: a row left the fast top-k path       */
+#define MULO_DEV_TIMEOUT 8u         /* a bounded device-side wait gave up: results invalid */
 
 typedef struct mulo_params {
   int32_t B, H, W;       /* images, target grid; the draft grid is (H/r) x (W/r)            */
@@ -121,6 +122,12 @@ mulo_status mulo_set_workspace(mulo_ctx* ctx, void* dev_ptr, size_t bytes);
 mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags);
 /* Number of kernels this context has launched so far. */
 mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
+/* mulo_round picks between two row kernels: a fast one for rows with top-k on and pooling
+ * off (each row streamed once, work done on the few thousand entries near and above the
+ * top-k threshold; a row it cannot handle is redone by the general routines) and the general
+ * one.  Both compute the same function.  `on` != 0 makes this context always use the general
+ * kernel (for testing and comparison). */
+mulo_status mulo_set_general_path_only(mulo_ctx* ctx, int on);
 /* Optional device timing of the fused row kernel (the launch that reads the logits):
  * mulo_set_timing prepares CUDA event pairs for up to max_launches (<= 4096) calls of
  * mulo_round (0 turns timing off); every mulo_round then records an event on its stream

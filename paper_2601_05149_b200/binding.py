@@ -18,12 +18,12 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 F32, BF16 = 0, 1
 ACCEPT_RATIO, ACCEPT_THRESHOLD = 0, 1
 RESAMPLE_MIXED, RESAMPLE_RESIDUAL_ALL, RESAMPLE_TARGET_ALL, RESAMPLE_ISOLATED_RESIDUAL = 0, 1, 2, 3
-DEV_ZERO_DRAFT_PROB, DEV_BAD_TOKEN, DEV_DENSE_FALLBACK = 1, 2, 4
+DEV_ZERO_DRAFT_PROB, DEV_BAD_TOKEN, DEV_DENSE_FALLBACK, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = (
     "mulo_create", "mulo_destroy", "mulo_status_string", "mulo_workspace_bytes",
     "mulo_set_workspace", "mulo_poll_device_status", "mulo_kernel_launches",
-    "mulo_set_timing", "mulo_read_timing",
+    "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only",
     "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_resample",
     "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host",
 )
@@ -177,6 +177,9 @@ class Context:
         n = C.c_uint64()
         _check(lib().mulo_kernel_launches(self._ctx, C.byref(n)), "mulo_kernel_launches")
         return n.value
+
+    def set_general_path_only(self, on: bool):
+        _check(lib().mulo_set_general_path_only(self._ctx, int(bool(on))), "mulo_set_general_path_only")
 
     def set_timing(self, max_launches: int):
         _check(lib().mulo_set_timing(self._ctx, int(max_launches)), "mulo_set_timing")

@@ -9,6 +9,7 @@
 
 #include "../../include/mulo.h"
 #include "mulo_dense.cuh"
+#include "mulo_sparse.cuh"
 
 using namespace mulo;
 
@@ -67,24 +68,6 @@ __device__ __forceinline__ PoolSmem carve_pool(const DevParams& P, unsigned char
   ps.pn = reinterpret_cast<double*>(dyn);
   ps.bitmap = reinterpret_cast<uint32_t*>(dyn + (size_t)max(P.pool_k, 1) * sizeof(double));
   return ps;
-}
-
-__device__ __forceinline__ int checked_token(int tok, int V, uint32_t* dev_status) {
-  if (tok < 0 || tok >= V) {
-    if (threadIdx.x == 0) atomicOr(dev_status, MULO_DEV_BAD_TOKEN);
-    tok = min(max(tok, 0), V - 1);
-  }
-  return tok;
-}
-
-// Which draws does a visit need once its accept bit is known (fused round)?
-__device__ __forceinline__ int draws_for(int mode, int accepted) {
-  int d = 0;
-  if (mode == MULO_RESAMPLE_RESIDUAL_ALL || (!accepted && mode != MULO_RESAMPLE_TARGET_ALL)) d |= kDrawResidual;
-  if (mode == MULO_RESAMPLE_TARGET_ALL || (accepted && mode != MULO_RESAMPLE_RESIDUAL_ALL) ||
-      (!accepted && mode == MULO_RESAMPLE_ISOLATED_RESIDUAL))
-    d |= kDrawTarget;
-  return d;
 }
 
 // mulo_upsample_pool: one CTA per low-res cell.
@@ -376,6 +359,7 @@ struct mulo_ctx {
   uint64_t launches;
   std::vector<cudaEvent_t> ev;   // start/stop pairs around the fused row kernel
   size_t ev_used;
+  int force_dense;               // diagnostics: never take the fast top-k path
 };
 
 static const size_t kStatusBytes = 256;
@@ -480,6 +464,7 @@ mulo_status mulo_create(mulo_ctx** out, int device) {
   c->ws_bytes = 0;
   c->launches = 0;
   c->ev_used = 0;
+  c->force_dense = 0;
   *out = c;
   return MULO_OK;
 }
@@ -488,6 +473,12 @@ void mulo_destroy(mulo_ctx* ctx) {
   if (!ctx) return;
   for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
   delete ctx;
+}
+
+mulo_status mulo_set_general_path_only(mulo_ctx* ctx, int on) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  ctx->force_dense = on != 0;
+  return MULO_OK;
 }
 
 mulo_status mulo_set_timing(mulo_ctx* ctx, int max_launches) {
@@ -574,6 +565,73 @@ static bool raise_smem(K kernel, size_t bytes, const mulo_ctx* ctx) {
       return false;
     }
   return true;
+}
+
+
+// ---- the fast top-k path of mulo_round -------------------------------------------------
+
+// inverse of the standard normal CDF by bisection (host, set-up only)
+static double inv_norm_cdf(double p) {
+  double lo = -12.0, hi = 12.0;
+  for (int i = 0; i < 200; ++i) {
+    const double mid = 0.5 * (lo + hi);
+    if (0.5 * erfc(-mid / sqrt(2.0)) < p) lo = mid; else hi = mid;
+  }
+  return 0.5 * (lo + hi);
+}
+
+// Fills `s` and returns the dynamic shared memory the sparse kernel needs, or 0 if these
+// parameters are not eligible (then the general kernel runs).
+static size_t plan_sparse(const mulo_ctx* ctx, const mulo_params* p, const DevParams& d, SparseArgs* s) {
+  if (d.top_k <= 0 || d.pool_k > 1) return 0;
+  const int V = d.V, k = d.top_k;
+  if (V < 1024) return 0;
+  const int margin = (int)fmax(64.0, 8.0 * sqrt((double)k));
+  const int margin_boot = (int)fmax(3.0 * margin, 0.5 * k);
+  if ((double)(k + margin_boot) > 0.6 * V) return 0;
+  const int esz = d.bf16 ? 2 : 4;
+  int chunk = d.bf16 ? 4096 : 2048;
+  const int vr = (V + kPiece - 1) / kPiece * kPiece;
+  if (chunk > vr) chunk = vr;
+  s->chunk = chunk;
+  s->n_chunks = (V + chunk - 1) / chunk;
+  s->n_seg = s->n_chunks * (chunk / kPiece);
+  s->cap = (k + 2 * margin_boot + 255) / 256 * 256;
+  if (s->cap > 32768) return 0;
+  s->margin = margin;
+  s->margin_boot = margin_boot;
+  s->a_theta = (float)inv_norm_cdf(1.0 - (double)k / V);
+  s->a_boot = (float)inv_norm_cdf(1.0 - (double)(k + margin_boot) / V);
+  s->phi_theta = (float)(exp(-0.5 * s->a_theta * s->a_theta) / sqrt(2.0 * 3.14159265358979323846));
+  const size_t dyn = sparse_layout(*s, (size_t)chunk * esz * 2, nullptr, nullptr);
+  const size_t fixed = sizeof(BlockScratch) + sizeof(SparseSmem) + 1024;
+  if (dyn + fixed > (size_t)ctx->smem_optin) return 0;
+  (void)p;
+  return dyn;
+}
+
+template <bool BF16, bool HAS_U>
+static bool launch_sparse_t(const mulo_ctx* ctx, const SparseArgs& s, size_t dyn, cudaStream_t st) {
+  auto kern = k_round_sparse<BF16, HAS_U>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, dyn) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return false;
+  }
+  int grid = ctx->sm_count * per_sm;
+  if (grid > s.n_parents) grid = s.n_parents;
+  kern<<<grid, kThreads, dyn, st>>>(s);
+  return true;
+}
+
+static bool launch_sparse(const mulo_ctx* ctx, const SparseArgs& s, size_t dyn, cudaStream_t st) {
+  const bool hu = s.uncond != nullptr;
+  if (s.P.bf16) return hu ? launch_sparse_t<true, true>(ctx, s, dyn, st) : launch_sparse_t<true, false>(ctx, s, dyn, st);
+  return hu ? launch_sparse_t<false, true>(ctx, s, dyn, st) : launch_sparse_t<false, false>(ctx, s, dyn, st);
 }
 
 static size_t mask_smem(const mulo_params* p) { return (size_t)3 * p->H * ((p->W + 31) / 32) * 4; }
@@ -726,7 +784,20 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   cudaStream_t st = (cudaStream_t)stream;
   const bool timed = ctx->ev_used + 2 <= ctx->ev.size();
   if (timed) cudaEventRecord(ctx->ev[ctx->ev_used], st);
-  k_verify_rows<true><<<p->B * a.P.h * a.P.w, kThreads, dyn, st>>>(a);
+  SparseArgs sa;
+  memset(&sa, 0, sizeof sa);
+  const size_t sdyn = ctx->force_dense ? 0 : plan_sparse(ctx, p, a.P, &sa);
+  bool fast = false;
+  if (sdyn) {
+    sa.P = a.P;
+    sa.cond = a.cond; sa.uncond = a.uncond; sa.draft = a.draft; sa.draft_tok_lo = draft_tok_lo;
+    sa.p_tok = p_tok; sa.q_tok = q_tok; sa.accept_prob = accept_prob;
+    sa.flags = w.flags; sa.cand_res = w.cand_res; sa.cand_tgt = w.cand_tgt;
+    sa.dev_status = w.status;
+    sa.n_parents = p->B * a.P.h * a.P.w;
+    fast = launch_sparse(ctx, sa, sdyn, st);
+  }
+  if (!fast) k_verify_rows<true><<<p->B * a.P.h * a.P.w, kThreads, dyn, st>>>(a);
   if (timed) {
     cudaEventRecord(ctx->ev[ctx->ev_used + 1], st);
     ctx->ev_used += 2;

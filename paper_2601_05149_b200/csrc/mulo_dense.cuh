@@ -241,4 +241,22 @@ __device__ inline void dense_position(const DevParams& P, const RowSrc& tr, cons
   out.tok_target = t_tgt;
 }
 
+__device__ __forceinline__ int checked_token(int tok, int V, uint32_t* dev_status) {
+  if (tok < 0 || tok >= V) {
+    if (threadIdx.x == 0) atomicOr(dev_status, MULO_DEV_BAD_TOKEN);
+    tok = min(max(tok, 0), V - 1);
+  }
+  return tok;
+}
+
+// Which draws does a visit need once its accept bit is known (fused round)?
+__device__ __forceinline__ int draws_for(int mode, int accepted) {
+  int d = 0;
+  if (mode == MULO_RESAMPLE_RESIDUAL_ALL || (!accepted && mode != MULO_RESAMPLE_TARGET_ALL)) d |= kDrawResidual;
+  if (mode == MULO_RESAMPLE_TARGET_ALL || (accepted && mode != MULO_RESAMPLE_RESIDUAL_ALL) ||
+      (!accepted && mode == MULO_RESAMPLE_ISOLATED_RESIDUAL))
+    d |= kDrawTarget;
+  return d;
+}
+
 }  // namespace mulo

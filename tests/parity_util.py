@@ -146,6 +146,8 @@ def check_round(cfg, g, oracle_out, prob_rtol=None):
         excused += e
         flagged += f
     total = len(oracle_out) * cfg.H * cfg.W
-    assert flagged <= max(1, int(1e-4 * total)) or flagged / total < 1e-4, (flagged, total)
+    # `flagged` is what the oracle marked as borderline (for an inverse-CDF draw over n
+    # active tokens that is a 2e-6 * n slice of the unit interval, so it is not small);
+    # the budget below is on positions where the GPU actually differed and was excused.
     assert excused <= max(1, int(1e-4 * total)) or excused / total < 1e-4, (excused, total)
     return excused, flagged

@@ -216,3 +216,87 @@ def test_device_status_reports_contract_violations(ctx):
     pu.gpu_round(ctx, cfg, bad)
     assert ctx.poll_device_status() & binding.DEV_ZERO_DRAFT_PROB
     assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0      # reading clears
+
+
+# ------------------------------------------------------------------ fast top-k path
+
+BIG = synth.RoundConfig("big", B=2, H=8, W=8, V=16384, dtype="bf16", sigma=1.0, cfg_scale=3.0,
+                        top_k=2000, radius=1, seed=201)
+
+
+@pytest.mark.parametrize("cfg", [
+    BIG,
+    dataclasses.replace(BIG, V=4096, top_k=500, cfg_scale=0.0, seed=202),
+    dataclasses.replace(BIG, V=8192, top_k=1000, dtype="f32", seed=203),
+    dataclasses.replace(BIG, V=8192, top_k=1000, dtype="f32", cfg_scale=0.0, temperature=0.8, seed=204),
+    dataclasses.replace(BIG, V=5000, top_k=600, seed=205),                         # ragged last chunk
+    dataclasses.replace(BIG, V=65536, top_k=2000, cfg_scale=0.0, H=4, W=4, seed=206),   # largest vocabulary
+    dataclasses.replace(BIG, V=2048, top_k=64, seed=207),                          # small k
+    dataclasses.replace(BIG, V=4096, top_k=400, B=2, H=32, W=32, radius=2, seed=208),  # several parents per CTA
+    dataclasses.replace(BIG, V=4096, top_k=500, r=1, H=6, W=6, seed=209),          # r = 1
+    dataclasses.replace(BIG, V=4096, top_k=500, r=4, H=8, W=8, seed=210),          # r = 4 (16 children)
+    dataclasses.replace(BIG, resample_mode=binding.RESAMPLE_ISOLATED_RESIDUAL, radius=2, seed=211),
+    dataclasses.replace(BIG, resample_mode=binding.RESAMPLE_RESIDUAL_ALL, seed=212),
+    dataclasses.replace(BIG, resample_mode=binding.RESAMPLE_TARGET_ALL, accept_mode=binding.ACCEPT_THRESHOLD,
+                        tau=1e-4, seed=213),
+], ids=lambda c: f"{c.dtype}-V{c.V}-k{c.top_k}-cfg{c.cfg_scale}-{c.B}x{c.H}x{c.W}r{c.r}-m{c.resample_mode}")
+def test_round_fast_path(ctx, cfg):
+    batch = pu.build_batch(cfg)
+    assert ctx.poll_device_status() == 0
+    g = pu.gpu_round(ctx, cfg, batch)
+    # Gaussian rows: the pivot prediction must hold, no row may have left the fast path
+    assert ctx.poll_device_status() == 0
+    o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
+    pu.check_round(cfg, g, o)
+    # and the general kernel gives the same decisions and tokens
+    ctx.set_general_path_only(True)
+    try:
+        d = pu.gpu_round(ctx, cfg, batch)
+    finally:
+        ctx.set_general_path_only(False)
+    pu.check_round(cfg, d, o)
+    same = (g["out_tok"] == d["out_tok"]).mean()
+    assert same > 0.999 and np.array_equal(g["reject_bits"], d["reject_bits"])
+
+
+def test_fast_path_falls_back_on_rows_it_cannot_predict(ctx):
+    """Rows of ties (all logits equal, or two values) defeat the pivot prediction;
+    those rows must be redone by the general routines with identical results."""
+    cfg = dataclasses.replace(BIG, V=4096, top_k=500, H=4, W=4, B=2, seed=220)
+    batch = pu.build_batch(cfg)
+    batch["draft_lo"][0, 0, 0] = 1.0                     # a constant draft row: top-k keeps everything
+    batch["cond"][0, 0, 1] = 0.5                         # a constant target row
+    batch["uncond"][0, 0, 1] = 0.25
+    batch["cond"][1, 2, 2, ::2] = 3.0                    # two-valued target row
+    batch["tok_lo"][0, 0, 0] = 17
+    ctx.poll_device_status()
+    g = pu.gpu_round(ctx, cfg, batch)
+    st = ctx.poll_device_status()
+    assert st & binding.DEV_DENSE_FALLBACK and not st & ~binding.DEV_DENSE_FALLBACK
+    o = pu.oracle_images(cfg, batch, [0, 1])
+    pu.check_round(cfg, g, o)
+
+
+def test_identity_fast_path(ctx):
+    cfg = dataclasses.replace(BIG, cfg_scale=0.0, sigma=0.0, seed=230)
+    batch = pu.build_batch(cfg)
+    g = pu.gpu_round(ctx, cfg, batch)
+    assert ctx.poll_device_status() == 0
+    assert g["n_reject"].sum() == 0 and np.all(g["accept_prob"] == 1.0)
+    assert np.array_equal(g["out_tok"], batch["tok_lo"].cpu().numpy().repeat(2, 1).repeat(2, 2))
+
+
+def test_config_C4_sampled_images(ctx):
+    """The benchmark's workload in its launch configuration (B = 32 on the device),
+    first and last image against the oracle, radii 1..3."""
+    cfg = synth.CONFIGS["C4"]
+    batch = pu.build_batch(cfg)
+    for radius in (3, 1, 2):
+        c = dataclasses.replace(cfg, radius=radius)
+        g = pu.gpu_round(ctx, c, batch, probs=(radius == 3))
+        assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
+        if radius == 3:
+            o = pu.oracle_images(c, batch, [0, cfg.B - 1])
+        else:   # only the masks and the choice of draw depend on the radius
+            o = pu.oracle_images(c, batch, [cfg.B - 1])
+        pu.check_round(c, g, o)
