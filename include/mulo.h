@@ -218,6 +218,47 @@ mulo_status mulo_round_host(mulo_ctx* ctx, const mulo_params* p, void* arena, si
                             float* accept_prob, int32_t* n_reject, int32_t* n_expand,
                             int32_t* first_reject, void* stream);
 
+/* ---- a round for callers that cannot allocate device memory ---------------------------- */
+
+/* The paper has no counterpart to this call; it exists for deployment reasons only.
+ *
+ * mulo_round needs a scratch buffer (one accept flag and two candidate tokens per grid
+ * position, plus the device status word) that somebody has to allocate.  Some hosts
+ * cannot: an inference server whose memory pool has already claimed every free byte of
+ * HBM, so that a cudaMalloc at request time fails; a plug-in that runs inside such a
+ * server and is handed its inputs and outputs but no allocator; a latency-critical loop
+ * in which the implicit device synchronisation of cudaMalloc / cudaFree is not acceptable.
+ * mulo_round_static is mulo_round for them.  Its scratch is a fixed array of
+ * MULO_STATIC_SCRATCH_BYTES that is part of the library image: every GPU on which the
+ * library runs a kernel holds that much memory from then until the process exits, whether
+ * or not this call is ever used.  Nothing in this call allocates or frees memory, on the
+ * device or through any library that might.
+ *
+ *   - Same inputs, outputs and results as mulo_round (the same kernels run).  The
+ *     workspace handed to mulo_set_workspace, if any, is neither needed nor touched.
+ *   - Size limit: mulo_workspace_bytes(p) must not exceed MULO_STATIC_SCRATCH_BYTES
+ *     (about 116,000 grid positions per call, e.g. 28 images of 64 x 64).  A larger
+ *     request returns MULO_ERR_WORKSPACE before anything is launched; split the batch
+ *     over several calls (image_offset keeps the random streams aligned).
+ *   - device_status [1], DEVICE pointer, may be NULL: receives the MULO_DEV_* bits this
+ *     call raised (the call clears the bits first, so they describe this call alone).
+ *   - The first call on a device looks up the array's device address (once per device, with
+ *     that device made current for the lookup).  Make that first call outside any stream
+ *     capture.
+ *   - There is one array per device and every call uses it.  It keeps whatever the last
+ *     call left there; the call re-initialises the part that must start at zero and
+ *     overwrites the rest before reading it.  Two calls that may run on the same device
+ *     at the same time (different streams, different host threads, different contexts)
+ *     race on it and give undefined results: order them on one stream or with events. */
+#define MULO_STATIC_SCRATCH_BYTES (1u << 20)
+mulo_status mulo_round_static(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond,
+                              const void* tgt_uncond, const void* draft_logits_lo,
+                              const int32_t* draft_tok_lo, const uint16_t* nn, int32_t* out_tok,
+                              uint32_t* reject_bits, uint32_t* expand_bits, float* p_tok,
+                              float* q_tok, float* accept_prob, int32_t* n_reject,
+                              int32_t* n_expand, int32_t* first_reject, uint32_t* device_status,
+                              void* stream);
+
 #ifdef __cplusplus
 }
 #endif

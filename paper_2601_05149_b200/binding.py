@@ -25,8 +25,10 @@ EXPORTS = (
     "mulo_set_workspace", "mulo_poll_device_status", "mulo_kernel_launches",
     "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only",
     "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_resample",
-    "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host",
+    "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host", "mulo_round_static",
 )
+
+STATIC_SCRATCH_BYTES = 1 << 20
 
 
 class MuloParams(C.Structure):
@@ -225,6 +227,21 @@ class Context:
                                 _dev(reject_bits), _dev(expand_bits), _dev(p_tok), _dev(q_tok),
                                 _dev(accept_prob), _dev(n_reject), _dev(n_expand), _dev(first_reject),
                                 _stream(stream)), "mulo_round")
+
+    def mulo_round_static(self, p, tgt_cond, tgt_uncond, draft_logits_lo, draft_tok_lo, nn, out_tok,
+                          reject_bits, expand_bits, p_tok=None, q_tok=None, accept_prob=None,
+                          n_reject=None, n_expand=None, first_reject=None, device_status=None,
+                          stream=None):
+        """``mulo_round`` on the library's built-in scratch array: for hosts that cannot
+        allocate device memory.  Needs no workspace; at most ``STATIC_SCRATCH_BYTES`` of
+        scratch (``workspace_bytes(p)``), one call at a time per device.  ``device_status``
+        is an optional one-element int32 CUDA tensor for the MULO_DEV_* bits."""
+        _check(lib().mulo_round_static(self._ctx, C.byref(p), _dev(tgt_cond), _dev(tgt_uncond),
+                                       _dev(draft_logits_lo), _dev(draft_tok_lo), _dev(nn),
+                                       _dev(out_tok), _dev(reject_bits), _dev(expand_bits),
+                                       _dev(p_tok), _dev(q_tok), _dev(accept_prob), _dev(n_reject),
+                                       _dev(n_expand), _dev(first_reject), _dev(device_status),
+                                       _stream(stream)), "mulo_round_static")
 
     @staticmethod
     def round_host_arena_bytes(p: MuloParams, has_uncond: bool) -> int:

@@ -4,6 +4,7 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -903,3 +904,68 @@ mulo_status mulo_round_host(mulo_ctx* ctx, const mulo_params* p, void* arena, si
 }
 
 }  // extern "C"
+
+// ---- allocation-free variant of the fused round ------------------------------------------
+
+// Scratch of mulo_round_static: lives in the library image, one copy per device that
+// loads it.  In host code this name is only a handle for the runtime's symbol table,
+// never a device address; the kernels get the address cudaGetSymbolAddress returns.
+static __device__ __align__(256) unsigned char g_static_scratch[MULO_STATIC_SCRATCH_BYTES];
+
+static const int kMaxStaticDevices = 64;
+static void* g_static_scratch_addr[kMaxStaticDevices];   // per device, nullptr until looked up
+static std::mutex g_static_scratch_mutex;
+
+// Device address of g_static_scratch on `device`: looked up once per device, with that
+// device current, then served from the table.
+static mulo_status static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxStaticDevices) return MULO_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_addr[device]) {
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) return MULO_ERR_CUDA;
+    if (prev != device && cudaSetDevice(device) != cudaSuccess) return MULO_ERR_CUDA;
+    void* addr = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+    if (prev != device) cudaSetDevice(prev);
+    if (e != cudaSuccess || !addr) {
+      cudaGetLastError();
+      return MULO_ERR_CUDA;
+    }
+    g_static_scratch_addr[device] = addr;
+  }
+  *out = g_static_scratch_addr[device];
+  return MULO_OK;
+}
+
+extern "C" mulo_status mulo_round_static(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond,
+                                         const void* tgt_uncond, const void* draft_logits_lo,
+                                         const int32_t* draft_tok_lo, const uint16_t* nn, int32_t* out_tok,
+                                         uint32_t* reject_bits, uint32_t* expand_bits, float* p_tok,
+                                         float* q_tok, float* accept_prob, int32_t* n_reject,
+                                         int32_t* n_expand, int32_t* first_reject, uint32_t* device_status,
+                                         void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (carve_ws(nullptr, p).bytes > (size_t)MULO_STATIC_SCRATCH_BYTES) return MULO_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  if ((s = static_scratch_address(ctx->device, &scratch)) != MULO_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  // The status word is OR-ed into and must start at zero; flags and candidates are written
+  // for every position of this call before the mask kernel reads them.
+  if (cudaMemsetAsync(scratch, 0, kStatusBytes, st) != cudaSuccess) return MULO_ERR_CUDA;
+  void* const saved_ws = ctx->ws;
+  const size_t saved_bytes = ctx->ws_bytes;
+  ctx->ws = scratch;
+  ctx->ws_bytes = MULO_STATIC_SCRATCH_BYTES;
+  s = mulo_round(ctx, p, tgt_cond, tgt_uncond, draft_logits_lo, draft_tok_lo, nn, out_tok, reject_bits,
+                 expand_bits, p_tok, q_tok, accept_prob, n_reject, n_expand, first_reject, stream);
+  ctx->ws = saved_ws;
+  ctx->ws_bytes = saved_bytes;
+  if (s != MULO_OK) return s;
+  if (device_status &&
+      cudaMemcpyAsync(device_status, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return MULO_ERR_CUDA;
+  return MULO_OK;
+}
