@@ -232,6 +232,7 @@ def run_ours(args, cfg):
     n_rej = int(out["n_reject"].sum().item())
     n_exp = int(out["n_expand"].sum().item())
     status = ctx.poll_device_status()
+    fallback = ctx.poll_fallback_counts()
 
     # roofline of the row kernel: algorithmic bytes of one launch / its mean duration
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -242,7 +243,7 @@ def run_ours(args, cfg):
     alg_bytes = cfg.algorithmic_bytes_per_position() * positions
     row_avg_ms = row_ms / max(1, row_n)
     achieved = alg_bytes / (row_avg_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "k_verify_rows<fused>", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "k_round_stream", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                 "frac_of_nominal_8TBps": achieved / 8000.0, "traffic": None,
                 "bytes_per_launch": alg_bytes, "avg_launch_ms": row_avg_ms, "launches_timed": row_n}
@@ -271,7 +272,8 @@ def run_ours(args, cfg):
             "config": {"workload": workload_desc(cfg), "per_gpu_batch": cfg.B,
                        "l2": "inputs per step (%.2f GB) exceed the 126 MB L2; no flush needed" % (alg_bytes / 1e9),
                        "acceptance_rate": 1.0 - n_rej / positions, "expanded_fraction": n_exp / positions,
-                       "device_status": status},
+                       "device_status": status,
+                       "rows_redone_by_general_kernel": fallback[0], "fallback_reasons": fallback[1:]},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
         }))
     ctx.close()

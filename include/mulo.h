@@ -120,6 +120,15 @@ mulo_status mulo_workspace_bytes(const mulo_params* p, size_t* bytes);
 mulo_status mulo_set_workspace(mulo_ctx* ctx, void* dev_ptr, size_t bytes);
 /* Synchronises `stream`, reads and clears the device status bits (MULO_DEV_*). */
 mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags);
+/* Synchronises `stream`, reads and clears five counters kept next to the status bits:
+ * counts[0] rows that mulo_round's fast kernel handed to the general routines, and of those
+ * counts[1] because a candidate list was full, counts[2] because fewer than top_k candidates
+ * passed the predicted pivot, counts[3] because the k-th largest lay above the selection
+ * histogram, counts[4] because too many entries tied near it (the target rows under a draft
+ * row that was handed over follow it without a reason of their own).  Results are the same
+ * either way; a large counts[0] means the rows are far from what the predictor expects and
+ * the round runs at the general kernel's speed. */
+mulo_status mulo_poll_fallback_counts(mulo_ctx* ctx, void* stream, uint32_t counts[5]);
 /* Number of kernels this context has launched so far. */
 mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
 /* mulo_round picks between two row kernels: a fast one for rows with top-k on and pooling

@@ -22,7 +22,7 @@ DEV_ZERO_DRAFT_PROB, DEV_BAD_TOKEN, DEV_DENSE_FALLBACK, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = (
     "mulo_create", "mulo_destroy", "mulo_status_string", "mulo_workspace_bytes",
-    "mulo_set_workspace", "mulo_poll_device_status", "mulo_kernel_launches",
+    "mulo_set_workspace", "mulo_poll_device_status", "mulo_poll_fallback_counts", "mulo_kernel_launches",
     "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only",
     "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_resample",
     "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host", "mulo_round_static",
@@ -174,6 +174,13 @@ class Context:
         _check(lib().mulo_poll_device_status(self._ctx, _stream(stream), C.byref(f)),
                "mulo_poll_device_status")
         return f.value
+
+    def poll_fallback_counts(self, stream=None):
+        """[rows redone by the general routines, list full, too few candidates, k-th largest
+        above the histogram, crowded bin] since the last poll."""
+        c = (C.c_uint32 * 5)()
+        _check(lib().mulo_poll_fallback_counts(self._ctx, _stream(stream), c), "mulo_poll_fallback_counts")
+        return [int(x) for x in c]
 
     def kernel_launches(self) -> int:
         n = C.c_uint64()

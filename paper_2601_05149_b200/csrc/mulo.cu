@@ -10,7 +10,7 @@
 
 #include "../../include/mulo.h"
 #include "mulo_dense.cuh"
-#include "mulo_sparse.cuh"
+#include "mulo_stream.cuh"
 
 using namespace mulo;
 
@@ -536,6 +536,17 @@ mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags
   return MULO_OK;
 }
 
+mulo_status mulo_poll_fallback_counts(mulo_ctx* ctx, void* stream, uint32_t counts[5]) {
+  if (!ctx || !counts) return MULO_ERR_INVALID_ARG;
+  if (!ctx->ws) return MULO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* src = (char*)ctx->ws + sizeof(uint32_t);
+  if (cudaMemcpyAsync(counts, src, 5 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MULO_ERR_CUDA;
+  if (cudaMemsetAsync(src, 0, 5 * sizeof(uint32_t), st) != cudaSuccess) return MULO_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MULO_ERR_CUDA;
+  return MULO_OK;
+}
+
 mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count) {
   if (!ctx || !count) return MULO_ERR_INVALID_ARG;
   *count = ctx->launches;
@@ -581,39 +592,57 @@ static double inv_norm_cdf(double p) {
   return 0.5 * (lo + hi);
 }
 
-// Fills `s` and returns the dynamic shared memory the sparse kernel needs, or 0 if these
+// P(X > c) for X ~ binomial(n, p)
+static double binom_tail(int n, double p, int c) {
+  double pmf = pow(1.0 - p, n), cdf = 0.0;
+  for (int x = 0; x <= c && x <= n; ++x) {
+    cdf += pmf;
+    pmf *= (double)(n - x) / (x + 1) * p / (1.0 - p);
+  }
+  return fmax(0.0, 1.0 - cdf);
+}
+
+// Fills `s` and returns the dynamic shared memory the streaming kernel needs, or 0 if these
 // parameters are not eligible (then the general kernel runs).
-static size_t plan_sparse(const mulo_ctx* ctx, const mulo_params* p, const DevParams& d, SparseArgs* s) {
+static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s) {
   if (d.top_k <= 0 || d.pool_k > 1) return 0;
   const int V = d.V, k = d.top_k;
-  if (V < 1024) return 0;
-  const int margin = (int)fmax(64.0, 8.0 * sqrt((double)k));
-  const int margin_boot = (int)fmax(3.0 * margin, 0.5 * k);
-  if ((double)(k + margin_boot) > 0.6 * V) return 0;
+  if (V < 1024 || 1 + d.r * d.r > kMaxRowsPerParent) return 0;
+  // candidates aimed for beyond k: about six standard deviations of the count of entries
+  // above a fixed value near the k-th largest
+  const int margin = (int)fmax(64.0, 6.0 * sqrt((double)k));
+  const int margin_boot = 2 * margin;
+  if ((double)(k + margin_boot) > 0.5 * V) return 0;
   const int esz = d.bf16 ? 2 : 4;
-  int chunk = d.bf16 ? 4096 : 2048;
-  const int vr = (V + kPiece - 1) / kPiece * kPiece;
-  if (chunk > vr) chunk = vr;
-  s->chunk = chunk;
-  s->n_chunks = (V + chunk - 1) / chunk;
-  s->n_seg = s->n_chunks * (chunk / kPiece);
-  s->cap = (k + 2 * margin_boot + 255) / 256 * 256;
-  if (s->cap > 32768) return 0;
+  const int epl = 16 / esz, piece = 32 * epl;
+  s->chunk = kWarps * piece;
+  s->n_chunks = (V + s->chunk - 1) / s->chunk;
+  if (s->n_chunks > 255) return 0;
+  s->n_seg = s->n_chunks * kWarps;
+  // capacity of a segment's list: the smallest multiple of 8 that a binomial(piece, density)
+  // count exceeds, in any of a row's segments, with probability <= 1e-4 at the steady-state
+  // density and <= 2e-2 at the bootstrap density
+  int cap = 8;
+  for (; cap < piece; cap += 8)
+    if (s->n_seg * binom_tail(piece, (double)(k + margin) / V, cap) <= 1e-4 &&
+        s->n_seg * binom_tail(piece, (double)(k + margin_boot) / V, cap) <= 2e-2)
+      break;
+  if (cap > piece) cap = piece;
+  if (cap > 248) return 0;
+  s->cap = cap;
+  if ((size_t)s->n_seg * cap > 65535) return 0;
   s->margin = margin;
-  s->margin_boot = margin_boot;
   s->a_theta = (float)inv_norm_cdf(1.0 - (double)k / V);
   s->a_boot = (float)inv_norm_cdf(1.0 - (double)(k + margin_boot) / V);
-  s->phi_theta = (float)(exp(-0.5 * s->a_theta * s->a_theta) / sqrt(2.0 * 3.14159265358979323846));
-  const size_t dyn = sparse_layout(*s, (size_t)chunk * esz * 2, nullptr, nullptr);
-  const size_t fixed = sizeof(BlockScratch) + sizeof(SparseSmem) + 1024;
+  const size_t dyn = stream_layout(*s, esz);
+  const size_t fixed = sizeof(StreamSmem) + 1024;
   if (dyn + fixed > (size_t)ctx->smem_optin) return 0;
-  (void)p;
   return dyn;
 }
 
 template <bool BF16, bool HAS_U>
-static bool launch_sparse_t(const mulo_ctx* ctx, const SparseArgs& s, size_t dyn, cudaStream_t st) {
-  auto kern = k_round_sparse<BF16, HAS_U>;
+static bool launch_stream_t(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn, cudaStream_t st) {
+  auto kern = k_round_stream<BF16, HAS_U>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
     cudaGetLastError();
     return false;
@@ -629,10 +658,10 @@ static bool launch_sparse_t(const mulo_ctx* ctx, const SparseArgs& s, size_t dyn
   return true;
 }
 
-static bool launch_sparse(const mulo_ctx* ctx, const SparseArgs& s, size_t dyn, cudaStream_t st) {
+static bool launch_stream(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn, cudaStream_t st) {
   const bool hu = s.uncond != nullptr;
-  if (s.P.bf16) return hu ? launch_sparse_t<true, true>(ctx, s, dyn, st) : launch_sparse_t<true, false>(ctx, s, dyn, st);
-  return hu ? launch_sparse_t<false, true>(ctx, s, dyn, st) : launch_sparse_t<false, false>(ctx, s, dyn, st);
+  if (s.P.bf16) return hu ? launch_stream_t<true, true>(ctx, s, dyn, st) : launch_stream_t<true, false>(ctx, s, dyn, st);
+  return hu ? launch_stream_t<false, true>(ctx, s, dyn, st) : launch_stream_t<false, false>(ctx, s, dyn, st);
 }
 
 static size_t mask_smem(const mulo_params* p) { return (size_t)3 * p->H * ((p->W + 31) / 32) * 4; }
@@ -785,9 +814,9 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   cudaStream_t st = (cudaStream_t)stream;
   const bool timed = ctx->ev_used + 2 <= ctx->ev.size();
   if (timed) cudaEventRecord(ctx->ev[ctx->ev_used], st);
-  SparseArgs sa;
+  StreamArgs sa;
   memset(&sa, 0, sizeof sa);
-  const size_t sdyn = ctx->force_dense ? 0 : plan_sparse(ctx, p, a.P, &sa);
+  const size_t sdyn = ctx->force_dense ? 0 : plan_stream(ctx, a.P, &sa);
   bool fast = false;
   if (sdyn) {
     sa.P = a.P;
@@ -796,7 +825,7 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
     sa.flags = w.flags; sa.cand_res = w.cand_res; sa.cand_tgt = w.cand_tgt;
     sa.dev_status = w.status;
     sa.n_parents = p->B * a.P.h * a.P.w;
-    fast = launch_sparse(ctx, sa, sdyn, st);
+    fast = launch_stream(ctx, sa, sdyn, st);
   }
   if (!fast) k_verify_rows<true><<<p->B * a.P.h * a.P.w, kThreads, dyn, st>>>(a);
   if (timed) {

@@ -1,0 +1,1042 @@
+// The fast path of the fused round for rows with top-k on (no pooling).
+//
+// A persistent CTA owns a contiguous range of parent (low-res) cells.  For each
+// parent it streams the draft row and then its r*r target rows ONCE through a
+// shared-memory ring filled by bulk-async copies (cp.async.bulk + mbarrier); the
+// warp that releases a ring slot last requests the next chunk into it, so there
+// is no producer thread to wait for.  The streaming pass keeps only the entries
+// above a predicted pivot (k plus a margin) and writes them, in ascending token
+// id, into one fixed-capacity list per 32-lane piece of the row ("segment").
+// Everything else -- the exact k-th largest value, softmax, acceptance, residual
+// and the inverse-CDF draws -- works on those ~k candidates in shared memory.
+// Each warp post-processes the segments it wrote, eight lanes per segment, and
+// values every warp needs (threshold, partition sum, accept bit) are recomputed
+// by every warp from shared data instead of being broadcast behind a barrier.
+// A row whose prediction fails (too few candidates, a full segment, too many
+// ties at the threshold) is redone by the dense routines from global memory, so
+// results never depend on the prediction.
+//
+// State that is the same for all threads lives in shared memory or in the kernel
+// parameters, not in registers: two CTAs of 512 threads share an SM, which
+// leaves 64 registers per thread.
+#pragma once
+
+#include <type_traits>
+
+#include "mulo_dense.cuh"
+
+namespace mulo {
+
+// ------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// global -> shared bulk copy (16-byte aligned, size a multiple of 16), completion
+// counted in bytes on `bar`.  Never multicast.
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst_smem)),
+               "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+constexpr uint32_t kSpinLimit = 1u << 22;   // bounded waits: give up, flag, carry on
+
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return;
+  atomicOr(dev_status, MULO_DEV_TIMEOUT);   // the data is then garbage, but nothing hangs
+}
+
+// two fp32 operations per instruction (sm_100 packed fp32); each half is the
+// IEEE round-to-nearest result of the scalar operation
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+
+// exp(z - m) for the bulk of a row: a subtract, a multiply and one ex2.  Relative
+// error about 2^-22 (1 + |z - m|); the probability of the draft token itself,
+// which decides acceptance, is computed in double precision.
+__device__ __forceinline__ float fast_exp(float z, float m) {
+  float r;
+  const float t = __fmul_rn(__fsub_rn(z, m), 1.4426950408889634f);
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+  return r;
+}
+
+// ------------------------------------------------------------ configuration
+constexpr int kStages = 3;           // ring slots
+constexpr int kHistBins = 256;       // selection histogram bins
+constexpr int kMemberCap = 128;      // entries of the crossing bin ranked exactly
+constexpr int kSegLanes = 8;         // lanes that share one segment in the list passes
+constexpr int kSegGroups = 32 / kSegLanes;
+constexpr int kTableParents = 4;     // parents whose row addresses are kept
+constexpr int kMaxRowsPerParent = 17;   // draft row + r*r children, r <= 4
+// words of the device status block after the flag word: rows redone by the general
+// routines, and why the fast path gave them up
+enum : int { kCntRows = 1, kCntListFull = 2, kCntTooFew = 3, kCntAboveRange = 4, kCntCrowdedBin = 5 };
+
+struct StreamArgs {
+  DevParams P;
+  const char* cond;
+  const char* uncond;
+  const char* draft;
+  const int32_t* draft_tok_lo;
+  float* p_tok;
+  float* q_tok;
+  float* accept_prob;
+  uint8_t* flags;
+  int32_t* cand_res;
+  int32_t* cand_tgt;
+  uint32_t* dev_status;
+  int n_parents;
+  int chunk;        // elements per ring slot half = kWarps pieces
+  int n_chunks;     // chunks per row = ceil(V / chunk)
+  int n_seg;        // segments per row = n_chunks * kWarps; segment c * kWarps + w is warp w's piece of chunk c
+  int cap;          // candidate capacity per segment (multiple of 8, < 256)
+  int margin;       // extra candidates aimed for in steady state
+  float a_theta;    // Phi^-1(1 - k/V)
+  float a_boot;     // Phi^-1(1 - (k + bootstrap margin)/V)
+  // byte offsets into dynamic shared memory (computed on the host)
+  uint32_t slot_bytes, off_cand, off_qval, off_tcnt, off_qcnt, off_qcell, off_sega, off_segb, off_segc;
+};
+
+inline size_t stream_align(size_t x) { return (x + 127) / 128 * 128; }
+
+// Lays out dynamic shared memory; returns its size.  (host)
+inline size_t stream_layout(StreamArgs& a, int esz) {
+  const int epl = 16 / esz;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off += stream_align(bytes);
+    return (uint32_t)o;
+  };
+  const size_t n_list = (size_t)a.n_seg * a.cap;
+  a.slot_bytes = (uint32_t)((size_t)a.chunk * esz * 2);   // cond + uncond halves
+  take((size_t)a.slot_bytes * kStages);                   // the ring sits at offset 0
+  // uint2 (z, later e = exp(z - m); token id) of the target row.  The block-wide scratch of the
+  // bootstrap statistics and of the dense fallback lives here too: both run only while no
+  // target list is in use.
+  a.off_cand = take(n_list * 8 > sizeof(BlockScratch) ? n_list * 8 : sizeof(BlockScratch));
+  a.off_qval = take(n_list * 4);    // float z, later exp(z - m_q), of the draft row
+  a.off_tcnt = take((size_t)a.n_seg * 2);   // uint16 entries per segment, target row
+  a.off_qcnt = take((size_t)a.n_seg * 2);   // uint16 entries per segment, draft row
+  a.off_qcell = take((size_t)a.n_chunks * a.chunk / epl * 2);   // uint16 per lane visit of the draft row:
+                                                                // survivor mask | (first slot << 8)
+  a.off_sega = take((size_t)a.n_seg * 4);   // float per-segment sums of e without the threshold bin's entries
+  a.off_segb = take((size_t)a.n_seg * 4);   // float per-segment sums of residual weights
+  a.off_segc = take((size_t)a.n_seg * 4);   // float per-segment sums of e, complete
+  return off;
+}
+
+// Pivot predictor of one kind of row (draft rows / target rows), per CTA:
+// the running k-th largest value and the density of entries just below it.
+struct Predictor {
+  int have;
+  float theta, rho;
+};
+
+struct RowState {   // selection scratch of one row; two copies alternate between rows
+  unsigned hist[kHistBins];
+  float member_z[kMemberCap];
+  unsigned short member_at[kMemberCap];
+  unsigned short member_seg[kMemberCap];
+  unsigned n_cand, n_member, overflow, max_key;
+};
+
+struct RowPrep {    // per target row, prepared while the previous row is finished
+  uint32_t rnd[3];
+  float z_tok;      // pre-processed target logit of x~
+};
+
+struct StreamSmem {
+  uint64_t full[kStages];
+  unsigned done[kStages];
+  RowState rs[2];
+  RowPrep prep[2];
+  Predictor pred[2];   // 0: draft rows, 1: target rows
+  double e_tok;        // exp(z_tok - m_p) of the current target row
+  // the current parent
+  double Zq, q_tok;
+  float theta_q, m_q, invZq;
+  int q_ok, tok;
+  int b, ca, cc;
+  // the parent the address table was last filled for
+  int tb, tca, tcc, tparent;
+  unsigned long long row_off[kTableParents][kMaxRowsPerParent];   // byte offsets of the rows within their tensors
+};
+
+// Cursor of the next chunk to request: chunk within the row, row within the parent,
+// table slot of the parent.  Every thread carries the same copy and advances it once
+// per consumed chunk, so whichever warp is last out of a ring slot can issue.
+struct Cursor {
+  int left;          // chunks still to request
+  unsigned pos;      // c | j << 8 | table slot << 16
+};
+__device__ __forceinline__ void cursor_advance(Cursor& w, int n_chunks, int rows_per_parent) {
+  --w.left;
+  unsigned c = (w.pos & 0xffu) + 1u, j = (w.pos >> 8) & 0xffu, s = w.pos >> 16;
+  if (c == (unsigned)n_chunks) {
+    c = 0;
+    if (++j == (unsigned)rows_per_parent) {
+      j = 0;
+      s = (s + 1u) & (kTableParents - 1);
+    }
+  }
+  w.pos = c | (j << 8) | (s << 16);
+}
+
+template <bool BF16, bool HAS_U>
+__device__ __forceinline__ void cursor_issue(const Cursor& w, const StreamArgs& a, StreamSmem& sm,
+                                             unsigned char* ring, int slot) {
+  const int esz = BF16 ? 2 : 4;
+  const int c = (int)(w.pos & 0xffu), j = (int)((w.pos >> 8) & 0xffu), s = (int)(w.pos >> 16);
+  const int elems = min(a.chunk, a.P.V - c * a.chunk);
+  const uint32_t bytes = (uint32_t)elems * esz;
+  unsigned char* dst = ring + (size_t)slot * a.slot_bytes;
+  const size_t off = (size_t)sm.row_off[s][j] + (size_t)c * a.chunk * esz;
+  if (j == 0) {
+    mbar_expect_tx(&sm.full[slot], bytes);
+    bulk_load(dst, a.draft + off, bytes, &sm.full[slot]);
+  } else {
+    mbar_expect_tx(&sm.full[slot], HAS_U ? 2 * bytes : bytes);
+    bulk_load(dst, a.cond + off, bytes, &sm.full[slot]);
+    if (HAS_U) bulk_load(dst + (size_t)a.chunk * esz, a.uncond + off, bytes, &sm.full[slot]);
+  }
+}
+
+// Writes the row offsets of `parent` (coordinates b, ca, cc) into table slot s.
+__device__ __forceinline__ void table_fill(const StreamArgs& a, StreamSmem& sm, int s, int parent, int b, int ca,
+                                           int cc, int esz) {
+  const DevParams& P = a.P;
+  const size_t row = (size_t)P.V * esz;
+  sm.row_off[s][0] = (unsigned long long)((size_t)parent * row);
+  const size_t base = (size_t)b * P.H * P.W + (size_t)ca * P.r * P.W + (size_t)cc * P.r;
+  int j = 1;
+  for (int di = 0; di < P.r; ++di)
+    for (int dj = 0; dj < P.r; ++dj, ++j) sm.row_off[s][j] = (unsigned long long)((base + (size_t)di * P.W + dj) * row);
+}
+
+// EPL pre-processed logits of one lane from a ring slot (EPL = 16 bytes of the
+// conditional row: 8 bf16 or 4 fp32 entries)
+template <bool BF16, bool HAS_U>
+__device__ __forceinline__ void slot_load(const unsigned char* slot, int chunk_elems, int e, float s, float invT,
+                                          float (&z)[BF16 ? 8 : 4]) {
+  const bool scale = invT != 1.0f;
+  const uint64_t s2 = pack2(s, s), t2 = pack2(invT, invT);
+  if (BF16) {
+    const uint4 c = *reinterpret_cast<const uint4*>(slot + (size_t)e * 2);
+    uint4 u = make_uint4(0, 0, 0, 0);
+    if (HAS_U) u = *reinterpret_cast<const uint4*>(slot + (size_t)chunk_elems * 2 + (size_t)e * 2);
+    const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, uw[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint64_t v = pack2(bf16_lo(cw[i]), bf16_hi(cw[i]));
+      if (HAS_U) {
+        const uint64_t un = pack2(bf16_lo(uw[i]), bf16_hi(uw[i]));
+        v = fma2(s2, sub2(v, un), un);
+      }
+      if (scale) v = mul2(v, t2);
+      unpack2(v, z[2 * i], z[2 * i + 1]);
+    }
+  } else {
+    const float4 c = *reinterpret_cast<const float4*>(slot + (size_t)e * 4);
+    float4 u = make_float4(0, 0, 0, 0);
+    if (HAS_U) u = *reinterpret_cast<const float4*>(slot + (size_t)chunk_elems * 4 + (size_t)e * 4);
+    uint64_t v0 = pack2(c.x, c.y), v1 = pack2(c.z, c.w);
+    if (HAS_U) {
+      const uint64_t u0 = pack2(u.x, u.y), u1 = pack2(u.z, u.w);
+      v0 = fma2(s2, sub2(v0, u0), u0);
+      v1 = fma2(s2, sub2(v1, u1), u1);
+    }
+    if (scale) {
+      v0 = mul2(v0, t2);
+      v1 = mul2(v1, t2);
+    }
+    unpack2(v0, z[0], z[1]);
+    unpack2(v1, z[2], z[3]);
+  }
+}
+
+__device__ __forceinline__ float seg_lanes_sum(float v) {
+  v += __shfl_xor_sync(kFull, v, 1);
+  v += __shfl_xor_sync(kFull, v, 2);
+  v += __shfl_xor_sync(kFull, v, 4);
+  return v;
+}
+
+// First index within [0, cnt) of a segment whose running weight sum exceeds y
+// (one warp; weights from `wfun(i)`), or the last index with weight if rounding
+// leaves the sum short.  Returns -1 for an empty / weightless segment.
+template <class W>
+__device__ __forceinline__ int warp_locate(int cnt, float y, W wfun) {
+  const int lane = threadIdx.x & 31;
+  float carry = 0.f;
+  int last_pos = -1;
+  for (int base = 0; base < cnt; base += 32) {
+    const int i = base + lane;
+    float w = i < cnt ? wfun(i) : 0.f;
+    float inc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      float t = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const unsigned hit = __ballot_sync(kFull, w > 0.f && carry + inc > y);
+    if (hit) return base + __ffs(hit) - 1;
+    const unsigned pos = __ballot_sync(kFull, w > 0.f);
+    if (pos) last_pos = base + 31 - __clz(pos);
+    carry += __shfl_sync(kFull, inc, 31);
+  }
+  return last_pos;
+}
+
+// One inverse-CDF draw over per-segment weight sums `seg` (segments in ascending
+// token id, entries in ascending id inside a segment): scans the segment sums in
+// double, finds the segment that holds u * total, then the entry inside it.
+// Returns the index into the candidate array, or -1 when the total is zero.
+// Call from all lanes of ONE warp.
+template <class W>
+__device__ __forceinline__ int warp_draw(const float* seg, int n_seg, int cap, const uint16_t* cnt, double u,
+                                         W wfun) {
+  const int lane = threadIdx.x & 31;
+  double total = 0.0;
+  for (int s = lane; s < n_seg; s += 32) total += (double)seg[s];
+  total = warp_sum(total);
+  if (!(total > 0.0)) return -1;
+  const double y = u * total;
+  double carry = 0.0;
+  int last_seg = -1;
+  for (int base = 0; base < n_seg; base += 32) {
+    const int s = base + lane;
+    const double w = s < n_seg ? (double)seg[s] : 0.0;
+    double inc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      double t = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const unsigned hit = __ballot_sync(kFull, w > 0.0 && carry + inc > y);
+    if (hit) {
+      const int l = __ffs(hit) - 1;
+      const int sseg = base + l;
+      const double before = carry + __shfl_sync(kFull, inc - w, l);
+      const int at = warp_locate(min((int)cnt[sseg], cap), (float)(y - before),
+                                 [&](int i) { return wfun(sseg * cap + i); });
+      if (at >= 0) return sseg * cap + at;
+    }
+    const unsigned pos = __ballot_sync(kFull, w > 0.0);
+    if (pos) last_seg = base + 31 - __clz(pos);
+    carry += __shfl_sync(kFull, inc, 31);
+  }
+  if (last_seg < 0) return -1;
+  // rounding left u * total at (or past) the end: the last entry with weight
+  const int at = warp_locate(min((int)cnt[last_seg], cap), 3.0e38f, [&](int i) { return wfun(last_seg * cap + i); });
+  return at >= 0 ? last_seg * cap + at : -1;
+}
+
+// The dense routines, kept out of line so that the streaming kernel's register
+// allocation is not shaped by the rare path.
+__device__ __noinline__ void dense_fallback_position(const StreamArgs& a, StreamSmem& sm, size_t g, int t,
+                                                     uint32_t image, int parent, BlockScratch& bs) {
+  const DevParams& P = a.P;
+  const int esz = P.bf16 ? 2 : 4;
+  RowSrc tr = {a.cond + g * (size_t)P.V * esz, a.uncond ? a.uncond + g * (size_t)P.V * esz : nullptr, P.cfg_scale,
+               P.invT, P.V, P.bf16};
+  RowSrc qr = {a.draft + (size_t)parent * P.V * esz, nullptr, 0.f, P.invT, P.V, P.bf16};
+  RowStats sq = {sm.theta_q, sm.m_q, sm.Zq};
+  const int mode = P.resample_mode;
+  PoolSmem none = {nullptr, nullptr};
+  PositionOut o;
+  dense_position(P, tr, qr, sq, sm.tok, nullptr, image, (uint32_t)t, true, 0,
+                 [mode](int acc) { return draws_for(mode, acc); }, bs, none, a.dev_status, o);
+  if (threadIdx.x == 0) {
+    a.flags[g] = o.accepted ? 0 : 1;
+    a.cand_res[g] = o.tok_residual;
+    a.cand_tgt[g] = o.tok_target;
+    if (a.p_tok) a.p_tok[g] = o.p_tok;
+    if (a.q_tok) a.q_tok[g] = o.q_tok;
+    if (a.accept_prob) a.accept_prob[g] = o.accept_prob;
+  }
+}
+__device__ __noinline__ void dense_fallback_stats(const StreamArgs& a, StreamSmem& sm, int parent, BlockScratch& bs) {
+  const DevParams& P = a.P;
+  const int esz = P.bf16 ? 2 : 4;
+  RowSrc qr = {a.draft + (size_t)parent * P.V * esz, nullptr, 0.f, P.invT, P.V, P.bf16};
+  RowStats s;
+  dense_row_stats(qr, P.top_k, bs, s.theta, s.m, s.Z);
+  if (threadIdx.x == 0) {
+    sm.theta_q = s.theta;
+    sm.m_q = s.m;
+    sm.Zq = s.Z;
+  }
+}
+
+// where the k-th largest value lies in a row's selection histogram
+struct Sel {
+  int n;        // candidates streamed
+  int bstar;    // the histogram bin that holds the k-th largest
+  int want;     // its 1-based rank inside that bin, from below
+  int cum;      // entries in the bins below
+  float m;      // row maximum
+};
+
+template <bool BF16, bool HAS_U>
+__global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_constant__ StreamArgs a) {
+  constexpr int EPL = BF16 ? 8 : 4;        // entries per lane visit (16 bytes of the conditional row)
+  constexpr int PIECE = 32 * EPL;          // entries per warp visit = one segment
+  constexpr int esz = BF16 ? 2 : 4;
+  __shared__ StreamSmem sm;
+  extern __shared__ __align__(128) unsigned char dyn[];
+  const DevParams& P = a.P;
+  const int tid = threadIdx.x;
+#define MULO_LANE (tid & 31)
+#define MULO_WARP (tid >> 5)
+  unsigned char* const ring = dyn;
+  uint2* const cand = reinterpret_cast<uint2*>(dyn + a.off_cand);
+  float* const qval = reinterpret_cast<float*>(dyn + a.off_qval);
+  uint16_t* const tcnt = reinterpret_cast<uint16_t*>(dyn + a.off_tcnt);
+  uint16_t* const qcnt = reinterpret_cast<uint16_t*>(dyn + a.off_qcnt);
+  uint16_t* const qcell = reinterpret_cast<uint16_t*>(dyn + a.off_qcell);
+  float* const seg_a = reinterpret_cast<float*>(dyn + a.off_sega);
+  float* const seg_b = reinterpret_cast<float*>(dyn + a.off_segb);
+  float* const seg_c = reinterpret_cast<float*>(dyn + a.off_segc);
+  // block-wide scratch of the bootstrap statistics and the dense fallback: shares the
+  // target list's memory (never in use at the same time)
+  BlockScratch& bs = *reinterpret_cast<BlockScratch*>(dyn + a.off_cand);
+
+  // this CTA's parents: [p_begin, p_end)
+  const int p_begin = (int)(((long long)a.n_parents * blockIdx.x) / gridDim.x);
+  const int p_end = (int)(((long long)a.n_parents * (blockIdx.x + 1)) / gridDim.x);
+  if (p_end <= p_begin) return;
+  const int rows_per_parent = 1 + P.r * P.r;
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.full[s], 1);
+      sm.done[s] = 0;
+    }
+    mbar_fence_init();
+    for (int s = 0; s < 2; ++s) {
+      sm.rs[s].n_cand = 0;
+      sm.rs[s].n_member = 0;
+      sm.rs[s].overflow = 0;
+      sm.rs[s].max_key = 0;
+      sm.pred[s].have = 0;
+      sm.pred[s].theta = 0.f;
+      sm.pred[s].rho = 1.f;
+    }
+    const int hw = P.h * P.w;
+    sm.b = p_begin / hw;
+    sm.ca = (p_begin % hw) / P.w;
+    sm.cc = (p_begin % hw) % P.w;
+    // row addresses of the first three parents
+    int tb = sm.b, tca = sm.ca, tcc = sm.cc, tp = p_begin;
+    for (int i = 0; i < 3; ++i) {
+      if (tp < p_end) table_fill(a, sm, i, tp, tb, tca, tcc, esz);
+      if (i == 2) break;
+      ++tp;
+      if (++tcc == P.w) {
+        tcc = 0;
+        if (++tca == P.h) {
+          tca = 0;
+          ++tb;
+        }
+      }
+    }
+    sm.tb = tb;
+    sm.tca = tca;
+    sm.tcc = tcc;
+    sm.tparent = tp;
+  }
+  for (int i = tid; i < 2 * kHistBins; i += kThreads) sm.rs[i / kHistBins].hist[i % kHistBins] = 0;
+  __syncthreads();
+
+  Cursor cur;
+  cur.pos = 0;
+  cur.left = (p_end - p_begin) * rows_per_parent * a.n_chunks;
+  for (int s = 0; s < kStages && cur.left > 0; ++s) {
+    if (tid == 0) cursor_issue<BF16, HAS_U>(cur, a, sm, ring, s);
+    cursor_advance(cur, a.n_chunks, rows_per_parent);
+  }
+  int rslot = 0;          // ring slot of the next chunk to read
+  uint32_t rphase = 0;    // and its phase
+  int rowi = 0;           // rows streamed so far (selects the RowState / RowPrep copy)
+
+  // Releases the slot just read; the last warp out requests the next chunk into it.
+  auto release_slot = [&]() {
+    __syncwarp();
+    if (MULO_LANE == 0) {
+      __threadfence_block();
+      const unsigned old = atomicAdd(&sm.done[rslot], 1u);
+      if (old == (unsigned)kWarps - 1u) {
+        sm.done[rslot] = 0;
+        __threadfence_block();
+        if (cur.left > 0) cursor_issue<BF16, HAS_U>(cur, a, sm, ring, rslot);
+      }
+    }
+    if (cur.left > 0) cursor_advance(cur, a.n_chunks, rows_per_parent);
+    if (++rslot == kStages) {
+      rslot = 0;
+      rphase ^= 1u;
+    }
+  };
+
+  // Pivot and histogram scale of the next row of a kind.  Without a prediction the
+  // pivot is estimated from the mean and spread of the row's first chunk (which
+  // stays in its slot for the streaming pass).
+  auto choose_pivot = [&](int kind, auto has_u_tag, float& pivot, float& inv_w) {
+    constexpr bool ROW_U = decltype(has_u_tag)::value;
+    const Predictor pr = sm.pred[kind];
+    if (pr.have) {   // block-uniform
+      const float d = (float)a.margin / pr.rho;
+      pivot = pr.theta - d;
+      inv_w = (float)kHistBins / (3.0f * d);
+      return;
+    }
+    mbar_wait(&sm.full[rslot], rphase, a.dev_status);
+    const unsigned char* slot = ring + (size_t)rslot * a.slot_bytes;
+    const int elems = min(a.chunk, P.V);
+    float s1 = 0.f, s2 = 0.f;
+    for (int e = tid * EPL; e < elems; e += kThreads * EPL) {
+      float z[EPL];
+      slot_load<BF16, ROW_U>(slot, a.chunk, e, P.cfg_scale, P.invT, z);
+#pragma unroll
+      for (int j = 0; j < EPL; ++j) {
+        s1 += z[j];
+        s2 += z[j] * z[j];
+      }
+    }
+    const double S1 = block_sum((double)s1, bs), S2 = block_sum((double)s2, bs);
+    const float mean = (float)(S1 / elems);
+    const float sd = sqrtf(fmaxf((float)(S2 / elems) - mean * mean, 1e-20f));
+    const float d = fmaxf((a.a_theta - a.a_boot) * sd, 1e-20f);
+    pivot = mean + a.a_boot * sd;
+    inv_w = (float)kHistBins / (3.0f * d);
+  };
+
+  // Streams one row through the ring: entries with z >= pivot go, in ascending
+  // token id, to the fixed-capacity list of their segment.  Then (pass A) each
+  // warp histograms the low end of the lists it wrote and contributes to the
+  // row's maximum and candidate count.
+  auto stream_row = [&](auto is_q_tag, auto has_u_tag, float pivot, float inv_w, bool hist_pass) {
+    constexpr bool IS_Q = decltype(is_q_tag)::value;
+    constexpr bool ROW_U = decltype(has_u_tag)::value;
+    uint16_t* const cnt_arr = IS_Q ? qcnt : tcnt;
+    RowState& rs = sm.rs[rowi & 1];
+    const int lane = MULO_LANE, warp = MULO_WARP;
+    for (int c = 0; c < a.n_chunks; ++c) {
+      mbar_wait(&sm.full[rslot], rphase, a.dev_status);
+      const unsigned char* slot = ring + (size_t)rslot * a.slot_bytes;
+      const int e = warp * PIECE + lane * EPL;
+      const int id0 = c * a.chunk + e;
+      const int seg = c * kWarps + warp;
+      float z[EPL];
+      unsigned mask = 0;
+      if (id0 < P.V) {
+        slot_load<BF16, ROW_U>(slot, a.chunk, e, P.cfg_scale, P.invT, z);
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) mask |= (z[j] >= pivot ? 1u : 0u) << j;
+      }
+      const int cnt = __popc(mask);
+      int inc = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+      }
+      const int total = __shfl_sync(kFull, inc, 31);
+      const int off = inc - cnt;
+      if (lane == 31) cnt_arr[seg] = (uint16_t)total;
+      if (IS_Q && id0 < P.V) qcell[id0 / EPL] = (uint16_t)(mask | ((unsigned)min(off, 255) << 8));
+      if (total <= a.cap) {
+        if (IS_Q) {
+          float* dst = qval + seg * a.cap + off;
+#pragma unroll
+          for (int j = 0; j < EPL; ++j)
+            if ((mask >> j) & 1u) *dst++ = z[j];
+        } else {
+          uint2* dst = cand + seg * a.cap + off;
+#pragma unroll
+          for (int j = 0; j < EPL; ++j)
+            if ((mask >> j) & 1u) *dst++ = make_uint2(__float_as_uint(z[j]), (unsigned)(id0 + j));
+        }
+      } else if (lane == 0) {
+        rs.overflow = 1;
+      }
+      release_slot();
+    }
+    if (!hist_pass) return;   // block-uniform
+    __syncwarp();
+    const int sub = lane & (kSegLanes - 1);
+    float mx = -INFINITY;
+    unsigned mine = 0;
+    for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
+      const int c = c0 + lane / kSegLanes;
+      if (c < a.n_chunks) {
+        const int seg = c * kWarps + warp;
+        const int cn = min((int)cnt_arr[seg], a.cap);
+        if (sub == 0) mine += (unsigned)cn;
+        for (int sl = sub; sl < cn; sl += kSegLanes) {
+          const int at = seg * a.cap + sl;
+          const float z = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
+          mx = fmaxf(mx, z);
+          // (a full segment keeps entries of earlier rows, which may lie below the pivot:
+          // the row is redone anyway, but the index must stay inside the histogram)
+          const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
+          if (fb >= 0.f && fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+        }
+      }
+    }
+    __syncwarp();
+    const unsigned key = __reduce_max_sync(kFull, float_key(mx));
+    mine = __reduce_add_sync(kFull, mine);
+    if (lane == 0) {
+      atomicMax(&rs.max_key, key);
+      if (mine) atomicAdd(&rs.n_cand, mine);
+    }
+  };
+
+  // After the barrier that follows stream_row: where the k-th largest value lies in
+  // the histogram.  Every warp computes the same answer.  false: the row leaves the
+  // fast path (block-uniform).
+  auto locate_bin = [&](const RowState& rs, Sel& s) -> bool {
+    const int lane = MULO_LANE;
+    const int k = P.top_k;
+    s.n = (int)rs.n_cand;
+    if (rs.overflow || s.n < k) {
+      if (tid == 0) atomicAdd(a.dev_status + (rs.overflow ? kCntListFull : kCntTooFew), 1u);
+      return false;
+    }
+    s.m = key_float(rs.max_key);
+    const int rank = s.n - k + 1;   // 1-based rank from the bottom of the k-th largest
+    constexpr int PER = kHistBins / 32;
+    unsigned h[PER];
+    unsigned mine = 0;
+#pragma unroll
+    for (int b = 0; b < PER; ++b) {
+      h[b] = rs.hist[lane * PER + b];
+      mine += h[b];
+    }
+    unsigned inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned t = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const unsigned owner_mask = __ballot_sync(kFull, inc >= (unsigned)rank);
+    if (owner_mask == 0) {   // the rank lies above the histogram range
+      if (tid == 0) atomicAdd(a.dev_status + kCntAboveRange, 1u);
+      return false;
+    }
+    const int owner = __ffs(owner_mask) - 1;
+    unsigned cum = inc - mine, in_bin = 0;
+    int bstar = -1;
+#pragma unroll
+    for (int b = 0; b < PER; ++b) {
+      if (bstar < 0) {
+        if (cum + h[b] >= (unsigned)rank) {
+          bstar = lane * PER + b;
+          in_bin = h[b];
+        } else {
+          cum += h[b];
+        }
+      }
+    }
+    s.bstar = __shfl_sync(kFull, bstar, owner);
+    s.cum = (int)__shfl_sync(kFull, cum, owner);
+    in_bin = __shfl_sync(kFull, in_bin, owner);
+    s.want = rank - s.cum;
+    if (in_bin > (unsigned)kMemberCap) {
+      if (tid == 0) atomicAdd(a.dev_status + kCntCrowdedBin, 1u);
+      return false;
+    }
+    return true;
+  };
+
+  // Pass B over the warp's own segments: e = exp(z - m) for every entry at or above the
+  // crossing bin (0 below it); the bin's own entries are set aside to be ranked exactly
+  // and are left out of the segment sums for now.
+  auto exp_pass = [&](auto is_q_tag, RowState& rs, const Sel& s, float pivot, float inv_w) {
+    constexpr bool IS_Q = decltype(is_q_tag)::value;
+    const uint16_t* cnt_arr = IS_Q ? qcnt : tcnt;
+    const int lane = MULO_LANE, warp = MULO_WARP, sub = lane & (kSegLanes - 1);
+    for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
+      const int c = c0 + lane / kSegLanes;
+      const int seg = c * kWarps + warp;
+      float acc = 0.f;
+      if (c < a.n_chunks) {
+        const int cn = min((int)cnt_arr[seg], a.cap);
+        for (int sl = sub; sl < cn; sl += kSegLanes) {
+          const int at = seg * a.cap + sl;
+          const float z = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
+          const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
+          const int bin = fb < (float)kHistBins ? (int)fb : kHistBins;
+          float e = 0.f;
+          if (bin >= s.bstar) e = fast_exp(z, s.m);
+          if (bin == s.bstar) {
+            const unsigned slot = atomicAdd(&rs.n_member, 1u);
+            if (slot < (unsigned)kMemberCap) {
+              rs.member_z[slot] = z;
+              rs.member_at[slot] = (unsigned short)at;
+              rs.member_seg[slot] = (unsigned short)seg;
+            }
+          } else {
+            acc += e;
+          }
+          if (IS_Q) qval[at] = e;
+          else cand[at].x = __float_as_uint(e);
+        }
+      }
+      __syncwarp();
+      acc = seg_lanes_sum(acc);
+      if (sub == 0 && c < a.n_chunks) {
+        seg_a[seg] = acc;
+        if (!IS_Q) seg_c[seg] = acc;
+      }
+    }
+  };
+
+  // After the barrier that follows exp_pass: the exact k-th largest value theta, the
+  // number of entries >= theta, and the partition sum Z (every warp computes the same).
+  // Each warp also settles the set-aside entries that lie in its own segments: an entry
+  // below theta gets e = 0, one at or above it is added to the complete segment sum.
+  auto finish_selection = [&](auto is_q_tag, const RowState& rs, const Sel& s, float& theta, int& n_ge,
+                              double& Z) -> bool {
+    constexpr bool IS_Q = decltype(is_q_tag)::value;
+    const int lane = MULO_LANE, warp = MULO_WARP;
+    const int mcount = (int)rs.n_member;   // <= kMemberCap: locate_bin checked the bin's size
+    float th = 0.f;
+    int less_at = 0;
+    bool hit = false;
+    for (int i = lane; i < mcount; i += 32) {
+      const float vi = rs.member_z[i];
+      int less = 0, leq = 0;
+      for (int jj = 0; jj < mcount; ++jj) {
+        const float vj = rs.member_z[jj];
+        less += vj < vi;
+        leq += vj <= vi;
+      }
+      if (less < s.want && s.want <= leq) {
+        th = vi;
+        less_at = less;
+        hit = true;
+      }
+    }
+    __syncwarp();
+    const unsigned hm = __ballot_sync(kFull, hit);
+    if (hm == 0) return false;   // cannot happen: the bin holds the rank
+    const int src = __ffs(hm) - 1;
+    th = __shfl_sync(kFull, th, src);
+    less_at = __shfl_sync(kFull, less_at, src);
+    float zm = 0.f;
+    for (int i = lane; i < mcount; i += 32) {
+      const int at = rs.member_at[i], seg = rs.member_seg[i];
+      const bool keep = rs.member_z[i] >= th;
+      const bool own = (seg & (kWarps - 1)) == warp;   // one of this warp's segments
+      if (keep) {
+        const float e = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
+        zm += e;
+        if (own && !IS_Q) atomicAdd(&seg_c[seg], e);
+      } else if (own) {
+        if (IS_Q) qval[at] = 0.f;
+        else cand[at].x = 0u;
+      }
+    }
+    __syncwarp();
+    double z = (double)zm;
+    for (int sg = lane; sg < a.n_seg; sg += 32) z += (double)seg_a[sg];
+    Z = warp_sum(z);
+    theta = th;
+    n_ge = s.n - s.cum - less_at;
+    return true;
+  };
+
+  // Thread 0: the predictor of a kind of row after a row (ok: theta found exactly).
+  auto learn = [&](int kind, bool ok, float theta, float pivot, int n, int n_ge) {
+    Predictor pr = sm.pred[kind];
+    if (!ok) {
+      pr.have = 0;
+    } else {
+      const int below = n - n_ge;   // candidates in [pivot, theta)
+      float rho = pr.rho;
+      bool rho_ok = pr.have != 0;
+      if (theta > pivot && below >= 16) {
+        const float r_new = (float)below / (theta - pivot);
+        rho = pr.have ? pr.rho + 0.25f * (r_new - pr.rho) : r_new;
+        rho_ok = true;
+      }
+      if (!rho_ok) {   // no usable density yet: stay in bootstrap mode
+        pr.have = 0;
+      } else {
+        pr.theta = pr.have ? pr.theta + 0.25f * (theta - pr.theta) : theta;
+        pr.rho = rho;
+        pr.have = 1;
+      }
+    }
+    sm.pred[kind] = pr;
+  };
+
+  auto reset_state = [&](RowState& rs) {   // all threads; the copy must be idle
+    if (tid == 0) {
+      rs.n_cand = 0;
+      rs.n_member = 0;
+      rs.overflow = 0;
+      rs.max_key = 0;
+    }
+    if (tid < kHistBins) rs.hist[tid] = 0;
+  };
+
+  // One thread: the uniforms of a target position and the logit of x~ there.
+  auto prepare_row = [&](RowPrep& pp, int child) {
+    const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
+    const size_t g = (size_t)sm.b * P.H * P.W + t;
+    const uint4 r = philox4x32_10(make_uint4((uint32_t)t, (uint32_t)sm.b + P.image_offset, P.round, 0u),
+                                  make_uint2(P.seed_lo, P.seed_hi));
+    pp.rnd[0] = r.x;
+    pp.rnd[1] = r.y;
+    pp.rnd[2] = r.z;
+    RowSrc tr = {a.cond + g * (size_t)P.V * esz, HAS_U ? a.uncond + g * (size_t)P.V * esz : nullptr, P.cfg_scale,
+                 P.invT, P.V, BF16};
+    pp.z_tok = load1(tr, sm.tok);
+  };
+
+  for (int parent = p_begin; parent < p_end; ++parent) {
+    // ------------------------------------------------------------ draft row
+    {
+      if (tid == 0) {
+        sm.tok = checked_token(a.draft_tok_lo[parent], P.V, a.dev_status);
+        // row addresses two parents ahead
+        const int tp = sm.tparent + 1;
+        if (parent > p_begin && tp < p_end) {
+          int tb = sm.tb, tca = sm.tca, tcc = sm.tcc;
+          if (++tcc == P.w) {
+            tcc = 0;
+            if (++tca == P.h) {
+              tca = 0;
+              ++tb;
+            }
+          }
+          table_fill(a, sm, (tp - p_begin) & (kTableParents - 1), tp, tb, tca, tcc, esz);
+          sm.tb = tb;
+          sm.tca = tca;
+          sm.tcc = tcc;
+          sm.tparent = tp;
+        }
+      }
+      float pivot, inv_w;
+      choose_pivot(0, std::false_type{}, pivot, inv_w);
+      stream_row(std::true_type{}, std::false_type{}, pivot, inv_w, true);
+      RowState& rs = sm.rs[rowi & 1];
+      __syncthreads();
+      reset_state(sm.rs[(rowi + 1) & 1]);
+      Sel s;
+      bool ok = locate_bin(rs, s);
+      float theta = 0.f;
+      int n_ge = 0;
+      double Zq = 1.0;
+      if (ok) exp_pass(std::true_type{}, rs, s, pivot, inv_w);
+      __syncthreads();
+      if (ok) ok = finish_selection(std::true_type{}, rs, s, theta, n_ge, Zq);
+      if (tid == 0) {
+        learn(0, ok, theta, pivot, s.n, n_ge);
+        sm.q_ok = ok;
+        if (ok) {
+          sm.theta_q = theta;
+          sm.m_q = s.m;
+          sm.Zq = Zq;
+        } else {
+          atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
+          atomicAdd(a.dev_status + kCntRows, 1u);
+        }
+      }
+      if (!ok) {   // block-uniform
+        __syncthreads();
+        dense_fallback_stats(a, sm, parent, bs);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        // same rounding of Z_q as the unfused path (fp32 hi + lo)
+        const float Zhi = (float)sm.Zq, Zlo = (float)(sm.Zq - (double)Zhi);
+        const double Z = (double)Zhi + (double)Zlo;
+        RowSrc qr = {a.draft + (size_t)parent * P.V * esz, nullptr, 0.f, P.invT, P.V, BF16};
+        const float zq_tok = load1(qr, sm.tok);
+        const double q = (zq_tok >= sm.theta_q) ? exp((double)zq_tok - (double)sm.m_q) / Z : 0.0;
+        if (q <= 0.0) atomicOr(a.dev_status, MULO_DEV_ZERO_DRAFT_PROB);
+        sm.Zq = Z;
+        sm.q_tok = q;
+        sm.invZq = (float)(1.0 / Z);
+      }
+      if (tid == 64) prepare_row(sm.prep[(rowi + 1) & 1], 0);   // first child's uniforms and logit of x~
+      ++rowi;
+      __syncthreads();
+    }
+
+    // ------------------------------------------------------------ children
+    for (int child = 0; child < P.r * P.r; ++child) {
+      const bool q_ok = sm.q_ok != 0;
+      RowState& rs = sm.rs[rowi & 1];
+      const RowPrep& pp = sm.prep[rowi & 1];
+      float pivot, inv_w;
+      choose_pivot(1, std::integral_constant<bool, HAS_U>{}, pivot, inv_w);
+      stream_row(std::false_type{}, std::integral_constant<bool, HAS_U>{}, pivot, inv_w, q_ok);
+      __syncthreads();
+      reset_state(sm.rs[(rowi + 1) & 1]);
+      Sel s;
+      s.n = 0;
+      s.m = 0.f;
+      bool ok = q_ok && locate_bin(rs, s);
+      if (ok) {
+        if (tid == 32) sm.e_tok = exp((double)pp.z_tok - (double)s.m);
+        exp_pass(std::false_type{}, rs, s, pivot, inv_w);
+      }
+      __syncthreads();
+      float theta = 0.f;
+      int n_ge = 0;
+      double Zp = 1.0;
+      if (ok) ok = finish_selection(std::false_type{}, rs, s, theta, n_ge, Zp);
+      if (tid == 0 && q_ok) learn(1, ok, theta, pivot, s.n, n_ge);
+      const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
+      const size_t g = (size_t)sm.b * P.H * P.W + t;
+
+      if (ok) {
+        // ---- the decision (Eq. 1 / Eq. 5), the same in every warp
+        const double e_tok = (pp.z_tok >= theta) ? sm.e_tok : 0.0;
+        const double q_tok = sm.q_tok;
+        int accepted;
+        if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = e_tok >= P.tau * Zp;
+        else if (q_tok <= 0.0) accepted = e_tok > 0.0;
+        else accepted = uniform24(pp.rnd[0]) * q_tok * Zp < e_tok;
+        const int draws = draws_for(P.resample_mode, accepted);
+        const float invZp = (float)(1.0 / Zp), invZq = sm.invZq;
+        if (tid == 0) {
+          a.flags[g] = accepted ? 0 : 1;
+          if (a.p_tok) a.p_tok[g] = (float)(e_tok / Zp);
+          if (a.q_tok) a.q_tok[g] = (float)q_tok;
+          if (a.accept_prob) {
+            const double p = e_tok / Zp;
+            double thr;
+            if (P.accept_mode == MULO_ACCEPT_THRESHOLD) thr = p;
+            else if (q_tok <= 0.0) thr = p > 0.0 ? 1.0 : 0.0;
+            else thr = fmin(1.0, p / q_tok);
+            a.accept_prob[g] = (float)thr;
+          }
+        }
+        // weight of candidate i in the residual of Eq. 2 (lambda = 1)
+        auto w_resid = [&](int i) {
+          const uint2 en = cand[i];
+          const float pe = __fmul_rn(__uint_as_float(en.x), invZp);
+          const int id = (int)en.y;
+          const unsigned cell = qcell[id / EPL];
+          const int j = id % EPL;
+          float qe = 0.f;
+          if ((cell >> j) & 1u) qe = qval[(id / PIECE) * a.cap + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
+          return fmaxf(__fsub_rn(pe, __fmul_rn(qe, invZq)), 0.f);
+        };
+        auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
+        if (draws & kDrawResidual) {   // block-uniform
+          const int lane = MULO_LANE, warp = MULO_WARP, sub = lane & (kSegLanes - 1);
+          for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
+            const int c = c0 + lane / kSegLanes;
+            const int seg = c * kWarps + warp;
+            float acc = 0.f;
+            if (c < a.n_chunks) {
+              const int cn = min((int)tcnt[seg], a.cap);
+              for (int sl = sub; sl < cn; sl += kSegLanes) acc += w_resid(seg * a.cap + sl);
+            }
+            __syncwarp();
+            acc = seg_lanes_sum(acc);
+            if (sub == 0 && c < a.n_chunks) seg_b[seg] = acc;
+          }
+        }
+        __syncthreads();
+        const int warp = MULO_WARP;
+        if (warp == 0) {
+          int t_res = -1;
+          if (draws & kDrawResidual) {
+            int at = warp_draw(seg_b, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_resid);
+            if (at < 0)   // residual without mass: the target weights, same uniform
+              at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_target);
+            t_res = at >= 0 ? (int)cand[at].y : -1;
+          }
+          if (MULO_LANE == 0) a.cand_res[g] = t_res;
+        } else if (warp == 1) {
+          int t_tgt = -1;
+          if (draws & kDrawTarget) {
+            const int at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[2]), w_target);
+            t_tgt = at >= 0 ? (int)cand[at].y : -1;
+          }
+          if (MULO_LANE == 0) a.cand_tgt[g] = t_tgt;
+        } else if (tid == 64 && child + 1 < P.r * P.r) {
+          prepare_row(sm.prep[(rowi + 1) & 1], child + 1);
+        }
+      } else {
+        if (tid == 0) {
+          atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
+          atomicAdd(a.dev_status + kCntRows, 1u);
+        }
+        if (tid == 64 && child + 1 < P.r * P.r) prepare_row(sm.prep[(rowi + 1) & 1], child + 1);
+        __syncthreads();
+        dense_fallback_position(a, sm, g, t, (uint32_t)sm.b + P.image_offset, parent, bs);
+      }
+      ++rowi;
+      __syncthreads();
+    }
+    // next parent's coordinates (made visible by the barriers of its draft row)
+    if (tid == 0) {
+      if (++sm.cc == P.w) {
+        sm.cc = 0;
+        if (++sm.ca == P.h) {
+          sm.ca = 0;
+          ++sm.b;
+        }
+      }
+    }
+  }
+#undef MULO_LANE
+#undef MULO_WARP
+}
+
+}  // namespace mulo
