@@ -112,7 +112,8 @@ void mulo_destroy(mulo_ctx* ctx);
 const char* mulo_status_string(mulo_status s);
 
 /* Bytes of device scratch that calls with these parameters need (status word, per-position
- * accept flags and candidate tokens). */
+ * accept flags and candidate tokens, the list of positions the fast kernel leaves to the
+ * general routines): 13 bytes per grid position plus padding. */
 mulo_status mulo_workspace_bytes(const mulo_params* p, size_t* bytes);
 /* Hands the library a caller-owned device buffer (256-byte aligned).  It must stay valid
  * and must not be shared by calls that overlap on the device.  The first 256 bytes hold
@@ -246,7 +247,7 @@ mulo_status mulo_round_host(mulo_ctx* ctx, const mulo_params* p, void* arena, si
  *   - Same inputs, outputs and results as mulo_round (the same kernels run).  The
  *     workspace handed to mulo_set_workspace, if any, is neither needed nor touched.
  *   - Size limit: mulo_workspace_bytes(p) must not exceed MULO_STATIC_SCRATCH_BYTES
- *     (about 116,000 grid positions per call, e.g. 28 images of 64 x 64).  A larger
+ *     (about 80,000 grid positions per call, e.g. 19 images of 64 x 64).  A larger
  *     request returns MULO_ERR_WORKSPACE before anything is launched; split the batch
  *     over several calls (image_offset keeps the random streams aligned).
  *   - device_status [1], DEVICE pointer, may be NULL: receives the MULO_DEV_* bits this

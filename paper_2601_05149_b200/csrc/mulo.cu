@@ -161,6 +161,46 @@ __global__ void __launch_bounds__(kThreads) k_verify_rows(RowKernelArgs a) {
   }
 }
 
+// Second launch of mulo_round's fast path: the positions the streaming kernel put on its
+// list (rows whose pivot prediction failed), done by the dense routines, one CTA at a time.
+__global__ void __launch_bounds__(kThreads) k_verify_failed(RowKernelArgs a, const int32_t* fail_list,
+                                                            const uint32_t* fail_count) {
+  __shared__ BlockScratch bs;
+  const DevParams& P = a.P;
+  const int N = P.H * P.W;
+  const size_t total = (size_t)P.B * N;
+  const size_t n = min((size_t)*fail_count, total);
+  for (size_t idx = blockIdx.x; idx < n; idx += gridDim.x) {
+    const size_t g = (size_t)fail_list[idx];
+    if (g >= total) continue;
+    const int b = (int)(g / N), t = (int)(g % N), i = t / P.W, j = t % P.W;
+    const size_t cell = ((size_t)b * P.h + i / P.r) * P.w + j / P.r;
+    RowSrc qr = draft_row(a, cell);
+    RowStats sq;
+    dense_row_stats(qr, P.top_k, bs, sq.theta, sq.m, sq.Z);
+    {   // Z_q rounded as everywhere else (fp32 hi + lo)
+      const float Zhi = (float)sq.Z, Zlo = (float)(sq.Z - (double)Zhi);
+      sq.Z = (double)Zhi + (double)Zlo;
+    }
+    const int tok = checked_token(a.draft_tok_lo[cell], P.V, a.dev_status);
+    RowSrc tr = target_row(a, g);
+    PositionOut o;
+    const int mode = P.resample_mode;
+    PoolSmem none = {nullptr, nullptr};
+    dense_position(P, tr, qr, sq, tok, nullptr, (uint32_t)b + P.image_offset, (uint32_t)t, true, 0,
+                   [mode](int acc) { return draws_for(mode, acc); }, bs, none, a.dev_status, o);
+    if (threadIdx.x == 0) {
+      a.flags[g] = o.accepted ? 0 : 1;
+      a.cand_res[g] = o.tok_residual;
+      a.cand_tgt[g] = o.tok_target;
+      if (a.p_tok) a.p_tok[g] = o.p_tok;
+      if (a.q_tok) a.q_tok[g] = o.q_tok;
+      if (a.accept_prob) a.accept_prob[g] = o.accept_prob;
+    }
+    __syncthreads();
+  }
+}
+
 __device__ __forceinline__ int get_bit(const uint32_t* bits, int Ww, int H, int b, int i, int j) {
   return (bits[((size_t)b * H + i) * Ww + (j >> 5)] >> (j & 31)) & 1u;
 }
@@ -417,6 +457,7 @@ struct Workspace {
   uint8_t* flags;
   int32_t* cand_res;
   int32_t* cand_tgt;
+  int32_t* fail_list;   // positions the streaming kernel leaves to the dense routines
   size_t bytes;
 };
 
@@ -429,6 +470,7 @@ static Workspace carve_ws(void* base, const mulo_params* p) {
   w.flags = (uint8_t*)(c + off); off += align_up(n, 256);
   w.cand_res = (int32_t*)(c + off); off += align_up(n * 4, 256);
   w.cand_tgt = (int32_t*)(c + off); off += align_up(n * 4, 256);
+  w.fail_list = (int32_t*)(c + off); off += align_up(n * 4, 256);
   w.bytes = off;
   return w;
 }
@@ -615,10 +657,10 @@ static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s
   if ((double)(k + margin_boot) > 0.5 * V) return 0;
   const int esz = d.bf16 ? 2 : 4;
   const int epl = 16 / esz, piece = 32 * epl;
-  s->chunk = kWarps * piece;
+  s->chunk = kChunkPieces * piece;
   s->n_chunks = (V + s->chunk - 1) / s->chunk;
   if (s->n_chunks > 255) return 0;
-  s->n_seg = s->n_chunks * kWarps;
+  s->n_seg = s->n_chunks * kChunkPieces;
   // capacity of a segment's list: the smallest multiple of 8 that a binomial(piece, density)
   // count exceeds, in any of a row's segments, with probability <= 1e-4 at the steady-state
   // density and <= 2e-2 at the bootstrap density
@@ -648,13 +690,13 @@ static bool launch_stream_t(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn
     return false;
   }
   int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, dyn) != cudaSuccess || per_sm < 1) {
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kSThreads, dyn) != cudaSuccess || per_sm < 1) {
     cudaGetLastError();
     return false;
   }
   int grid = ctx->sm_count * per_sm;
   if (grid > s.n_parents) grid = s.n_parents;
-  kern<<<grid, kThreads, dyn, st>>>(s);
+  kern<<<grid, kSThreads, dyn, st>>>(s);
   return true;
 }
 
@@ -824,8 +866,12 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
     sa.p_tok = p_tok; sa.q_tok = q_tok; sa.accept_prob = accept_prob;
     sa.flags = w.flags; sa.cand_res = w.cand_res; sa.cand_tgt = w.cand_tgt;
     sa.dev_status = w.status;
+    sa.fail_list = w.fail_list;
     sa.n_parents = p->B * a.P.h * a.P.w;
+    if (cudaMemsetAsync(w.status + kFailCount, 0, sizeof(uint32_t), st) != cudaSuccess) return MULO_ERR_CUDA;
     fast = launch_stream(ctx, sa, sdyn, st);
+    // the rows the streaming kernel gave up on (usually a handful, often none)
+    if (fast) k_verify_failed<<<2 * ctx->sm_count, kThreads, 0, st>>>(a, w.fail_list, w.status + kFailCount);
   }
   if (!fast) k_verify_rows<true><<<p->B * a.P.h * a.P.w, kThreads, dyn, st>>>(a);
   if (timed) {
@@ -841,7 +887,7 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   m.cand_res = w.cand_res; m.cand_tgt = w.cand_tgt;
   m.draft_tok_lo = draft_tok_lo; m.out_tok = out_tok;
   k_mask<2><<<p->B, kMaskThreads, mask_smem(p), st>>>(m);
-  return launched(ctx, 2);
+  return launched(ctx, fast ? 3 : 2);
 }
 
 // ---- host-buffer variant -------------------------------------------------------------

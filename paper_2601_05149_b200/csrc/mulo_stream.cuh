@@ -1,24 +1,27 @@
 // The fast path of the fused round for rows with top-k on (no pooling).
 //
-// A persistent CTA owns a contiguous range of parent (low-res) cells.  For each
-// parent it streams the draft row and then its r*r target rows ONCE through a
-// shared-memory ring filled by bulk-async copies (cp.async.bulk + mbarrier); the
-// warp that releases a ring slot last requests the next chunk into it, so there
-// is no producer thread to wait for.  The streaming pass keeps only the entries
-// above a predicted pivot (k plus a margin) and writes them, in ascending token
-// id, into one fixed-capacity list per 32-lane piece of the row ("segment").
-// Everything else -- the exact k-th largest value, softmax, acceptance, residual
-// and the inverse-CDF draws -- works on those ~k candidates in shared memory.
-// Each warp post-processes the segments it wrote, eight lanes per segment, and
-// values every warp needs (threshold, partition sum, accept bit) are recomputed
-// by every warp from shared data instead of being broadcast behind a barrier.
-// A row whose prediction fails (too few candidates, a full segment, too many
-// ties at the threshold) is redone by the dense routines from global memory, so
-// results never depend on the prediction.
+// A persistent CTA (256 threads, two per SM) owns a contiguous range of parent
+// (low-res) cells.  For each parent it streams the draft row and then its r*r
+// target rows ONCE through a shared-memory ring of 32 KB slots filled by bulk-async
+// copies (cp.async.bulk + mbarrier); the warp that releases a slot last requests
+// the next chunk into it, so there is no producer thread to wait for.  A chunk
+// iteration has a fixed latency of several hundred cycles (barrier wait, shared
+// loads, release), so every warp works on four independent 32-lane pieces of the
+// row per iteration and releases the slot as soon as its data are in registers.
+// The streaming pass keeps only the entries above a predicted pivot (k plus a
+// margin) and writes them, in ascending token id, into one fixed-capacity list per
+// piece of the row ("segment").  Everything else -- the exact k-th largest value,
+// softmax, acceptance, residual and the inverse-CDF draws -- works on those ~k
+// candidates in shared memory.  Each warp post-processes the segments it wrote,
+// eight lanes per segment, and values every warp needs (threshold, partition sum,
+// accept bit) are recomputed by every warp from shared data instead of being
+// broadcast behind a barrier.  A row whose prediction fails (too few candidates, a
+// full segment, too many ties at the threshold) is put on a list that a second
+// launch works off with the dense routines, so results never depend on the
+// prediction and a failed row does not hold up its CTA.
 //
 // State that is the same for all threads lives in shared memory or in the kernel
-// parameters, not in registers: two CTAs of 512 threads share an SM, which
-// leaves 64 registers per thread.
+// parameters, not in registers.
 #pragma once
 
 #include <type_traits>
@@ -106,7 +109,11 @@ __device__ __forceinline__ float fast_exp(float z, float m) {
 }
 
 // ------------------------------------------------------------ configuration
-constexpr int kStages = 3;           // ring slots
+constexpr int kSThreads = 256;       // threads per CTA of the streaming kernel
+constexpr int kSWarps = kSThreads / 32;
+constexpr int kPPW = 4;              // pieces per warp per chunk (independent work per iteration)
+constexpr int kChunkPieces = kSWarps * kPPW;
+constexpr int kStages = 2;           // ring slots
 constexpr int kHistBins = 256;       // selection histogram bins
 constexpr int kMemberCap = 128;      // entries of the crossing bin ranked exactly
 constexpr int kSegLanes = 8;         // lanes that share one segment in the list passes
@@ -115,7 +122,8 @@ constexpr int kTableParents = 4;     // parents whose row addresses are kept
 constexpr int kMaxRowsPerParent = 17;   // draft row + r*r children, r <= 4
 // words of the device status block after the flag word: rows redone by the general
 // routines, and why the fast path gave them up
-enum : int { kCntRows = 1, kCntListFull = 2, kCntTooFew = 3, kCntAboveRange = 4, kCntCrowdedBin = 5 };
+enum : int { kCntRows = 1, kCntListFull = 2, kCntTooFew = 3, kCntAboveRange = 4, kCntCrowdedBin = 5,
+             kFailCount = 8 };   // word 8: length of the list of positions left to the dense routines
 
 struct StreamArgs {
   DevParams P;
@@ -130,16 +138,18 @@ struct StreamArgs {
   int32_t* cand_res;
   int32_t* cand_tgt;
   uint32_t* dev_status;
+  int32_t* fail_list;   // positions b*N + t whose rows the dense routines must do (length at dev_status[kFailCount])
   int n_parents;
-  int chunk;        // elements per ring slot half = kWarps pieces
+  int chunk;        // elements per ring slot half = kChunkPieces pieces
   int n_chunks;     // chunks per row = ceil(V / chunk)
-  int n_seg;        // segments per row = n_chunks * kWarps; segment c * kWarps + w is warp w's piece of chunk c
+  int n_seg;        // segments per row = n_chunks * kChunkPieces; segment c * kChunkPieces + p is piece p of
+                    // chunk c, handled by warp p % kSWarps
   int cap;          // candidate capacity per segment (multiple of 8, < 256)
   int margin;       // extra candidates aimed for in steady state
   float a_theta;    // Phi^-1(1 - k/V)
   float a_boot;     // Phi^-1(1 - (k + bootstrap margin)/V)
   // byte offsets into dynamic shared memory (computed on the host)
-  uint32_t slot_bytes, off_cand, off_qval, off_tcnt, off_qcnt, off_qcell, off_sega, off_segb, off_segc;
+  uint32_t slot_bytes, off_tz, off_tid, off_qval, off_tcnt, off_qcnt, off_qcell, off_sega, off_segb, off_segc;
 };
 
 inline size_t stream_align(size_t x) { return (x + 127) / 128 * 128; }
@@ -156,10 +166,8 @@ inline size_t stream_layout(StreamArgs& a, int esz) {
   const size_t n_list = (size_t)a.n_seg * a.cap;
   a.slot_bytes = (uint32_t)((size_t)a.chunk * esz * 2);   // cond + uncond halves
   take((size_t)a.slot_bytes * kStages);                   // the ring sits at offset 0
-  // uint2 (z, later e = exp(z - m); token id) of the target row.  The block-wide scratch of the
-  // bootstrap statistics and of the dense fallback lives here too: both run only while no
-  // target list is in use.
-  a.off_cand = take(n_list * 8 > sizeof(BlockScratch) ? n_list * 8 : sizeof(BlockScratch));
+  a.off_tz = take(n_list * 4);      // float z, later e = exp(z - m), of the target row's candidates
+  a.off_tid = take(n_list * 2);     // uint16 their token ids
   a.off_qval = take(n_list * 4);    // float z, later exp(z - m_q), of the draft row
   a.off_tcnt = take((size_t)a.n_seg * 2);   // uint16 entries per segment, target row
   a.off_qcnt = take((size_t)a.n_seg * 2);   // uint16 entries per segment, draft row
@@ -178,7 +186,7 @@ struct Predictor {
   float theta, rho;
 };
 
-struct RowState {   // selection scratch of one row; two copies alternate between rows
+struct RowState {   // selection scratch of the row in work
   unsigned hist[kHistBins];
   float member_z[kMemberCap];
   unsigned short member_at[kMemberCap];
@@ -194,9 +202,10 @@ struct RowPrep {    // per target row, prepared while the previous row is finish
 struct StreamSmem {
   uint64_t full[kStages];
   unsigned done[kStages];
-  RowState rs[2];
+  RowState rs;
   RowPrep prep[2];
   Predictor pred[2];   // 0: draft rows, 1: target rows
+  float red[kSWarps][2];   // bootstrap statistics
   double e_tok;        // exp(z_tok - m_p) of the current target row
   // the current parent
   double Zq, q_tok;
@@ -259,17 +268,23 @@ __device__ __forceinline__ void table_fill(const StreamArgs& a, StreamSmem& sm, 
     for (int dj = 0; dj < P.r; ++dj, ++j) sm.row_off[s][j] = (unsigned long long)((base + (size_t)di * P.W + dj) * row);
 }
 
-// EPL pre-processed logits of one lane from a ring slot (EPL = 16 bytes of the
-// conditional row: 8 bf16 or 4 fp32 entries)
+// 16 bytes of the conditional row (8 bf16 or 4 fp32 entries) of one lane, and the same
+// entries of the unconditional row, from a ring slot into registers
 template <bool BF16, bool HAS_U>
-__device__ __forceinline__ void slot_load(const unsigned char* slot, int chunk_elems, int e, float s, float invT,
-                                          float (&z)[BF16 ? 8 : 4]) {
+__device__ __forceinline__ void raw_load(const unsigned char* slot, int chunk_elems, int e, uint4& c, uint4& u) {
+  constexpr int esz = BF16 ? 2 : 4;
+  c = *reinterpret_cast<const uint4*>(slot + (size_t)e * esz);
+  u = make_uint4(0, 0, 0, 0);
+  if (HAS_U) u = *reinterpret_cast<const uint4*>(slot + (size_t)chunk_elems * esz + (size_t)e * esz);
+}
+// ... turned into pre-processed logits: d = c - u; v = fma(s, d, u); z = v * invT, each
+// one IEEE fp32 rounding (two entries per instruction)
+template <bool BF16, bool HAS_U>
+__device__ __forceinline__ void raw_mix(const uint4& c, const uint4& u, float s, float invT,
+                                        float (&z)[BF16 ? 8 : 4]) {
   const bool scale = invT != 1.0f;
   const uint64_t s2 = pack2(s, s), t2 = pack2(invT, invT);
   if (BF16) {
-    const uint4 c = *reinterpret_cast<const uint4*>(slot + (size_t)e * 2);
-    uint4 u = make_uint4(0, 0, 0, 0);
-    if (HAS_U) u = *reinterpret_cast<const uint4*>(slot + (size_t)chunk_elems * 2 + (size_t)e * 2);
     const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, uw[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -282,12 +297,9 @@ __device__ __forceinline__ void slot_load(const unsigned char* slot, int chunk_e
       unpack2(v, z[2 * i], z[2 * i + 1]);
     }
   } else {
-    const float4 c = *reinterpret_cast<const float4*>(slot + (size_t)e * 4);
-    float4 u = make_float4(0, 0, 0, 0);
-    if (HAS_U) u = *reinterpret_cast<const float4*>(slot + (size_t)chunk_elems * 4 + (size_t)e * 4);
-    uint64_t v0 = pack2(c.x, c.y), v1 = pack2(c.z, c.w);
+    uint64_t v0 = pack2(__uint_as_float(c.x), __uint_as_float(c.y)), v1 = pack2(__uint_as_float(c.z), __uint_as_float(c.w));
     if (HAS_U) {
-      const uint64_t u0 = pack2(u.x, u.y), u1 = pack2(u.z, u.w);
+      const uint64_t u0 = pack2(__uint_as_float(u.x), __uint_as_float(u.y)), u1 = pack2(__uint_as_float(u.z), __uint_as_float(u.w));
       v0 = fma2(s2, sub2(v0, u0), u0);
       v1 = fma2(s2, sub2(v1, u1), u1);
     }
@@ -377,43 +389,6 @@ __device__ __forceinline__ int warp_draw(const float* seg, int n_seg, int cap, c
   return at >= 0 ? last_seg * cap + at : -1;
 }
 
-// The dense routines, kept out of line so that the streaming kernel's register
-// allocation is not shaped by the rare path.
-__device__ __noinline__ void dense_fallback_position(const StreamArgs& a, StreamSmem& sm, size_t g, int t,
-                                                     uint32_t image, int parent, BlockScratch& bs) {
-  const DevParams& P = a.P;
-  const int esz = P.bf16 ? 2 : 4;
-  RowSrc tr = {a.cond + g * (size_t)P.V * esz, a.uncond ? a.uncond + g * (size_t)P.V * esz : nullptr, P.cfg_scale,
-               P.invT, P.V, P.bf16};
-  RowSrc qr = {a.draft + (size_t)parent * P.V * esz, nullptr, 0.f, P.invT, P.V, P.bf16};
-  RowStats sq = {sm.theta_q, sm.m_q, sm.Zq};
-  const int mode = P.resample_mode;
-  PoolSmem none = {nullptr, nullptr};
-  PositionOut o;
-  dense_position(P, tr, qr, sq, sm.tok, nullptr, image, (uint32_t)t, true, 0,
-                 [mode](int acc) { return draws_for(mode, acc); }, bs, none, a.dev_status, o);
-  if (threadIdx.x == 0) {
-    a.flags[g] = o.accepted ? 0 : 1;
-    a.cand_res[g] = o.tok_residual;
-    a.cand_tgt[g] = o.tok_target;
-    if (a.p_tok) a.p_tok[g] = o.p_tok;
-    if (a.q_tok) a.q_tok[g] = o.q_tok;
-    if (a.accept_prob) a.accept_prob[g] = o.accept_prob;
-  }
-}
-__device__ __noinline__ void dense_fallback_stats(const StreamArgs& a, StreamSmem& sm, int parent, BlockScratch& bs) {
-  const DevParams& P = a.P;
-  const int esz = P.bf16 ? 2 : 4;
-  RowSrc qr = {a.draft + (size_t)parent * P.V * esz, nullptr, 0.f, P.invT, P.V, P.bf16};
-  RowStats s;
-  dense_row_stats(qr, P.top_k, bs, s.theta, s.m, s.Z);
-  if (threadIdx.x == 0) {
-    sm.theta_q = s.theta;
-    sm.m_q = s.m;
-    sm.Zq = s.Z;
-  }
-}
-
 // where the k-th largest value lies in a row's selection histogram
 struct Sel {
   int n;        // candidates streamed
@@ -424,18 +399,18 @@ struct Sel {
 };
 
 template <bool BF16, bool HAS_U>
-__global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_constant__ StreamArgs a) {
+__global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_constant__ StreamArgs a) {
   constexpr int EPL = BF16 ? 8 : 4;        // entries per lane visit (16 bytes of the conditional row)
   constexpr int PIECE = 32 * EPL;          // entries per warp visit = one segment
   constexpr int esz = BF16 ? 2 : 4;
   __shared__ StreamSmem sm;
   extern __shared__ __align__(128) unsigned char dyn[];
   const DevParams& P = a.P;
-  const int tid = threadIdx.x;
-#define MULO_LANE (tid & 31)
-#define MULO_WARP (tid >> 5)
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane & (kSegLanes - 1), grp = lane / kSegLanes;
   unsigned char* const ring = dyn;
-  uint2* const cand = reinterpret_cast<uint2*>(dyn + a.off_cand);
+  float* const tz = reinterpret_cast<float*>(dyn + a.off_tz);
+  uint16_t* const tidl = reinterpret_cast<uint16_t*>(dyn + a.off_tid);
   float* const qval = reinterpret_cast<float*>(dyn + a.off_qval);
   uint16_t* const tcnt = reinterpret_cast<uint16_t*>(dyn + a.off_tcnt);
   uint16_t* const qcnt = reinterpret_cast<uint16_t*>(dyn + a.off_qcnt);
@@ -443,15 +418,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
   float* const seg_a = reinterpret_cast<float*>(dyn + a.off_sega);
   float* const seg_b = reinterpret_cast<float*>(dyn + a.off_segb);
   float* const seg_c = reinterpret_cast<float*>(dyn + a.off_segc);
-  // block-wide scratch of the bootstrap statistics and the dense fallback: shares the
-  // target list's memory (never in use at the same time)
-  BlockScratch& bs = *reinterpret_cast<BlockScratch*>(dyn + a.off_cand);
+  RowState& rs = sm.rs;
 
   // this CTA's parents: [p_begin, p_end)
   const int p_begin = (int)(((long long)a.n_parents * blockIdx.x) / gridDim.x);
   const int p_end = (int)(((long long)a.n_parents * (blockIdx.x + 1)) / gridDim.x);
   if (p_end <= p_begin) return;
-  const int rows_per_parent = 1 + P.r * P.r;
+  const int rr = P.r * P.r, rows_per_parent = 1 + rr;
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -459,11 +432,11 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
       sm.done[s] = 0;
     }
     mbar_fence_init();
+    rs.n_cand = 0;
+    rs.n_member = 0;
+    rs.overflow = 0;
+    rs.max_key = 0;
     for (int s = 0; s < 2; ++s) {
-      sm.rs[s].n_cand = 0;
-      sm.rs[s].n_member = 0;
-      sm.rs[s].overflow = 0;
-      sm.rs[s].max_key = 0;
       sm.pred[s].have = 0;
       sm.pred[s].theta = 0.f;
       sm.pred[s].rho = 1.f;
@@ -491,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
     sm.tcc = tcc;
     sm.tparent = tp;
   }
-  for (int i = tid; i < 2 * kHistBins; i += kThreads) sm.rs[i / kHistBins].hist[i % kHistBins] = 0;
+  if (tid < kHistBins) rs.hist[tid] = 0;
   __syncthreads();
 
   Cursor cur;
@@ -503,15 +476,15 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
   }
   int rslot = 0;          // ring slot of the next chunk to read
   uint32_t rphase = 0;    // and its phase
-  int rowi = 0;           // rows streamed so far (selects the RowState / RowPrep copy)
+  int rowi = 0;           // target rows done so far (selects the RowPrep copy)
 
   // Releases the slot just read; the last warp out requests the next chunk into it.
   auto release_slot = [&]() {
     __syncwarp();
-    if (MULO_LANE == 0) {
+    if (lane == 0) {
       __threadfence_block();
       const unsigned old = atomicAdd(&sm.done[rslot], 1u);
-      if (old == (unsigned)kWarps - 1u) {
+      if (old == (unsigned)kSWarps - 1u) {
         sm.done[rslot] = 0;
         __threadfence_block();
         if (cur.left > 0) cursor_issue<BF16, HAS_U>(cur, a, sm, ring, rslot);
@@ -540,16 +513,34 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
     const unsigned char* slot = ring + (size_t)rslot * a.slot_bytes;
     const int elems = min(a.chunk, P.V);
     float s1 = 0.f, s2 = 0.f;
-    for (int e = tid * EPL; e < elems; e += kThreads * EPL) {
+    for (int e = tid * EPL; e < elems; e += kSThreads * EPL) {
+      uint4 c, u;
       float z[EPL];
-      slot_load<BF16, ROW_U>(slot, a.chunk, e, P.cfg_scale, P.invT, z);
+      raw_load<BF16, ROW_U>(slot, a.chunk, e, c, u);
+      raw_mix<BF16, ROW_U>(c, u, P.cfg_scale, P.invT, z);
 #pragma unroll
       for (int j = 0; j < EPL; ++j) {
         s1 += z[j];
         s2 += z[j] * z[j];
       }
     }
-    const double S1 = block_sum((double)s1, bs), S2 = block_sum((double)s2, bs);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      s1 += __shfl_xor_sync(kFull, s1, o);
+      s2 += __shfl_xor_sync(kFull, s2, o);
+    }
+    if (lane == 0) {
+      sm.red[warp][0] = s1;
+      sm.red[warp][1] = s2;
+    }
+    __syncthreads();
+    double S1 = 0.0, S2 = 0.0;
+#pragma unroll
+    for (int w = 0; w < kSWarps; ++w) {
+      S1 += (double)sm.red[w][0];
+      S2 += (double)sm.red[w][1];
+    }
+    __syncthreads();
     const float mean = (float)(S1 / elems);
     const float sd = sqrtf(fmaxf((float)(S2 / elems) - mean * mean, 1e-20f));
     const float d = fmaxf((a.a_theta - a.a_boot) * sd, 1e-20f);
@@ -557,75 +548,109 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
     inv_w = (float)kHistBins / (3.0f * d);
   };
 
+  // Consumes a row's chunks without looking at them (a target row under a draft row
+  // that left the fast path).
+  auto skip_row = [&]() {
+    for (int c = 0; c < a.n_chunks; ++c) {
+      mbar_wait(&sm.full[rslot], rphase, a.dev_status);
+      release_slot();
+    }
+  };
+
   // Streams one row through the ring: entries with z >= pivot go, in ascending
   // token id, to the fixed-capacity list of their segment.  Then (pass A) each
   // warp histograms the low end of the lists it wrote and contributes to the
   // row's maximum and candidate count.
-  auto stream_row = [&](auto is_q_tag, auto has_u_tag, float pivot, float inv_w, bool hist_pass) {
+  auto stream_row = [&](auto is_q_tag, auto has_u_tag, float pivot, float inv_w) {
     constexpr bool IS_Q = decltype(is_q_tag)::value;
     constexpr bool ROW_U = decltype(has_u_tag)::value;
     uint16_t* const cnt_arr = IS_Q ? qcnt : tcnt;
-    RowState& rs = sm.rs[rowi & 1];
-    const int lane = MULO_LANE, warp = MULO_WARP;
     for (int c = 0; c < a.n_chunks; ++c) {
       mbar_wait(&sm.full[rslot], rphase, a.dev_status);
       const unsigned char* slot = ring + (size_t)rslot * a.slot_bytes;
-      const int e = warp * PIECE + lane * EPL;
-      const int id0 = c * a.chunk + e;
-      const int seg = c * kWarps + warp;
-      float z[EPL];
-      unsigned mask = 0;
-      if (id0 < P.V) {
-        slot_load<BF16, ROW_U>(slot, a.chunk, e, P.cfg_scale, P.invT, z);
+      uint4 rc[kPPW], ru[kPPW];
 #pragma unroll
-        for (int j = 0; j < EPL; ++j) mask |= (z[j] >= pivot ? 1u : 0u) << j;
+      for (int i = 0; i < kPPW; ++i) {
+        const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
+        if (c * a.chunk + e < P.V) raw_load<BF16, ROW_U>(slot, a.chunk, e, rc[i], ru[i]);
       }
-      const int cnt = __popc(mask);
-      int inc = cnt;
+      release_slot();   // the data are in registers
+      unsigned mask[kPPW];
+      float z[kPPW][EPL];
+#pragma unroll
+      for (int i = 0; i < kPPW; ++i) {
+        const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
+        mask[i] = 0;
+        if (c * a.chunk + e < P.V) {
+          raw_mix<BF16, ROW_U>(rc[i], ru[i], P.cfg_scale, P.invT, z[i]);
+#pragma unroll
+          for (int j = 0; j < EPL; ++j) mask[i] |= (z[i][j] >= pivot ? 1u : 0u) << j;
+        }
+      }
+      int cnt[kPPW], inc[kPPW];
+#pragma unroll
+      for (int i = 0; i < kPPW; ++i) inc[i] = cnt[i] = __popc(mask[i]);
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(kFull, inc, o);
-        if (lane >= o) inc += t;
-      }
-      const int total = __shfl_sync(kFull, inc, 31);
-      const int off = inc - cnt;
-      if (lane == 31) cnt_arr[seg] = (uint16_t)total;
-      if (IS_Q && id0 < P.V) qcell[id0 / EPL] = (uint16_t)(mask | ((unsigned)min(off, 255) << 8));
-      if (total <= a.cap) {
-        if (IS_Q) {
-          float* dst = qval + seg * a.cap + off;
 #pragma unroll
-          for (int j = 0; j < EPL; ++j)
-            if ((mask >> j) & 1u) *dst++ = z[j];
-        } else {
-          uint2* dst = cand + seg * a.cap + off;
-#pragma unroll
-          for (int j = 0; j < EPL; ++j)
-            if ((mask >> j) & 1u) *dst++ = make_uint2(__float_as_uint(z[j]), (unsigned)(id0 + j));
+        for (int i = 0; i < kPPW; ++i) {
+          const int t = __shfl_up_sync(kFull, inc[i], o);
+          if (lane >= o) inc[i] += t;
         }
-      } else if (lane == 0) {
-        rs.overflow = 1;
       }
-      release_slot();
+#pragma unroll
+      for (int i = 0; i < kPPW; ++i) {
+        const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
+        const int id0 = c * a.chunk + e;
+        const int seg = c * kChunkPieces + i * kSWarps + warp;
+        const int total = __shfl_sync(kFull, inc[i], 31);
+        const int off = inc[i] - cnt[i];
+        if (lane == 31) cnt_arr[seg] = (uint16_t)total;
+        if (IS_Q && id0 < P.V) qcell[id0 / EPL] = (uint16_t)(mask[i] | ((unsigned)min(off, 255) << 8));
+        if (total <= a.cap) {
+          if (IS_Q) {
+            float* dst = qval + seg * a.cap + off;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j)
+              if ((mask[i] >> j) & 1u) *dst++ = z[i][j];
+          } else {
+            float* dz = tz + seg * a.cap + off;
+            uint16_t* di = tidl + seg * a.cap + off;
+#pragma unroll
+            for (int j = 0; j < EPL; ++j)
+              if ((mask[i] >> j) & 1u) {
+                *dz++ = z[i][j];
+                *di++ = (uint16_t)(id0 + j);
+              }
+          }
+        } else if (lane == 0) {
+          rs.overflow = 1;
+        }
+      }
     }
-    if (!hist_pass) return;   // block-uniform
+    // ---- pass A over the lists this warp wrote: group `grp` of 8 lanes takes piece grp of each chunk
     __syncwarp();
-    const int sub = lane & (kSegLanes - 1);
+    float* const val = IS_Q ? qval : tz;
     float mx = -INFINITY;
     unsigned mine = 0;
-    for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
-      const int c = c0 + lane / kSegLanes;
-      if (c < a.n_chunks) {
-        const int seg = c * kWarps + warp;
-        const int cn = min((int)cnt_arr[seg], a.cap);
-        if (sub == 0) mine += (unsigned)cn;
-        for (int sl = sub; sl < cn; sl += kSegLanes) {
-          const int at = seg * a.cap + sl;
-          const float z = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
-          mx = fmaxf(mx, z);
-          // (a full segment keeps entries of earlier rows, which may lie below the pivot:
-          // the row is redone anyway, but the index must stay inside the histogram)
-          const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
+    for (int c0 = 0; c0 < a.n_chunks; c0 += 2) {
+      const int segA = c0 * kChunkPieces + grp * kSWarps + warp, segB = segA + kChunkPieces;
+      const int cnA = min((int)cnt_arr[segA], a.cap);
+      const int cnB = c0 + 1 < a.n_chunks ? min((int)cnt_arr[segB], a.cap) : 0;
+      if (sub == 0) mine += (unsigned)(cnA + cnB);
+      for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
+        // (a full segment keeps entries of earlier rows, which may lie below the pivot: the row is
+        // redone anyway, but the index must stay inside the histogram)
+        if (sl < cnA) {
+          const float zz = val[segA * a.cap + sl];
+          mx = fmaxf(mx, zz);
+          const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
+          if (fb >= 0.f && fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+        }
+        if (sl < cnB) {
+          const float zz = val[segB * a.cap + sl];
+          mx = fmaxf(mx, zz);
+          const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
           if (fb >= 0.f && fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
         }
       }
@@ -642,8 +667,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
   // After the barrier that follows stream_row: where the k-th largest value lies in
   // the histogram.  Every warp computes the same answer.  false: the row leaves the
   // fast path (block-uniform).
-  auto locate_bin = [&](const RowState& rs, Sel& s) -> bool {
-    const int lane = MULO_LANE;
+  auto locate_bin = [&](Sel& s) -> bool {
     const int k = P.top_k;
     s.n = (int)rs.n_cand;
     if (rs.overflow || s.n < k) {
@@ -699,42 +723,49 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
   // Pass B over the warp's own segments: e = exp(z - m) for every entry at or above the
   // crossing bin (0 below it); the bin's own entries are set aside to be ranked exactly
   // and are left out of the segment sums for now.
-  auto exp_pass = [&](auto is_q_tag, RowState& rs, const Sel& s, float pivot, float inv_w) {
+  auto exp_pass = [&](auto is_q_tag, const Sel& s, float pivot, float inv_w) {
     constexpr bool IS_Q = decltype(is_q_tag)::value;
     const uint16_t* cnt_arr = IS_Q ? qcnt : tcnt;
-    const int lane = MULO_LANE, warp = MULO_WARP, sub = lane & (kSegLanes - 1);
-    for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
-      const int c = c0 + lane / kSegLanes;
-      const int seg = c * kWarps + warp;
-      float acc = 0.f;
-      if (c < a.n_chunks) {
-        const int cn = min((int)cnt_arr[seg], a.cap);
-        for (int sl = sub; sl < cn; sl += kSegLanes) {
-          const int at = seg * a.cap + sl;
-          const float z = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
-          const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
-          const int bin = fb < (float)kHistBins ? (int)fb : kHistBins;
-          float e = 0.f;
-          if (bin >= s.bstar) e = fast_exp(z, s.m);
-          if (bin == s.bstar) {
-            const unsigned slot = atomicAdd(&rs.n_member, 1u);
-            if (slot < (unsigned)kMemberCap) {
-              rs.member_z[slot] = z;
-              rs.member_at[slot] = (unsigned short)at;
-              rs.member_seg[slot] = (unsigned short)seg;
-            }
-          } else {
-            acc += e;
-          }
-          if (IS_Q) qval[at] = e;
-          else cand[at].x = __float_as_uint(e);
+    float* const val = IS_Q ? qval : tz;
+    auto one = [&](int seg, int sl, float& acc) {
+      const int at = seg * a.cap + sl;
+      const float z = val[at];
+      const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
+      const int bin = fb < (float)kHistBins ? (int)fb : kHistBins;
+      float e = 0.f;
+      if (bin >= s.bstar) e = fast_exp(z, s.m);
+      if (bin == s.bstar) {
+        const unsigned slot = atomicAdd(&rs.n_member, 1u);
+        if (slot < (unsigned)kMemberCap) {
+          rs.member_z[slot] = z;
+          rs.member_at[slot] = (unsigned short)at;
+          rs.member_seg[slot] = (unsigned short)seg;
         }
+      } else {
+        acc += e;
+      }
+      val[at] = e;
+    };
+    for (int c0 = 0; c0 < a.n_chunks; c0 += 2) {
+      const int segA = c0 * kChunkPieces + grp * kSWarps + warp, segB = segA + kChunkPieces;
+      const bool hasB = c0 + 1 < a.n_chunks;
+      const int cnA = min((int)cnt_arr[segA], a.cap);
+      const int cnB = hasB ? min((int)cnt_arr[segB], a.cap) : 0;
+      float accA = 0.f, accB = 0.f;
+      for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
+        if (sl < cnA) one(segA, sl, accA);
+        if (sl < cnB) one(segB, sl, accB);
       }
       __syncwarp();
-      acc = seg_lanes_sum(acc);
-      if (sub == 0 && c < a.n_chunks) {
-        seg_a[seg] = acc;
-        if (!IS_Q) seg_c[seg] = acc;
+      accA = seg_lanes_sum(accA);
+      accB = seg_lanes_sum(accB);
+      if (sub == 0) {
+        seg_a[segA] = accA;
+        if (!IS_Q) seg_c[segA] = accA;
+        if (hasB) {
+          seg_a[segB] = accB;
+          if (!IS_Q) seg_c[segB] = accB;
+        }
       }
     }
   };
@@ -743,10 +774,9 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
   // number of entries >= theta, and the partition sum Z (every warp computes the same).
   // Each warp also settles the set-aside entries that lie in its own segments: an entry
   // below theta gets e = 0, one at or above it is added to the complete segment sum.
-  auto finish_selection = [&](auto is_q_tag, const RowState& rs, const Sel& s, float& theta, int& n_ge,
-                              double& Z) -> bool {
+  auto finish_selection = [&](auto is_q_tag, const Sel& s, float& theta, int& n_ge, double& Z) -> bool {
     constexpr bool IS_Q = decltype(is_q_tag)::value;
-    const int lane = MULO_LANE, warp = MULO_WARP;
+    float* const val = IS_Q ? qval : tz;
     const int mcount = (int)rs.n_member;   // <= kMemberCap: locate_bin checked the bin's size
     float th = 0.f;
     int less_at = 0;
@@ -771,22 +801,20 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
     const int src = __ffs(hm) - 1;
     th = __shfl_sync(kFull, th, src);
     less_at = __shfl_sync(kFull, less_at, src);
-    float zm = 0.f;
+    double z = 0.0;
     for (int i = lane; i < mcount; i += 32) {
       const int at = rs.member_at[i], seg = rs.member_seg[i];
       const bool keep = rs.member_z[i] >= th;
-      const bool own = (seg & (kWarps - 1)) == warp;   // one of this warp's segments
+      const bool own = (seg & (kSWarps - 1)) == warp;   // one of this warp's segments
       if (keep) {
-        const float e = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
-        zm += e;
+        const float e = val[at];
+        z += (double)e;
         if (own && !IS_Q) atomicAdd(&seg_c[seg], e);
       } else if (own) {
-        if (IS_Q) qval[at] = 0.f;
-        else cand[at].x = 0u;
+        val[at] = 0.f;
       }
     }
     __syncwarp();
-    double z = (double)zm;
     for (int sg = lane; sg < a.n_seg; sg += 32) z += (double)seg_a[sg];
     Z = warp_sum(z);
     theta = th;
@@ -819,7 +847,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
     sm.pred[kind] = pr;
   };
 
-  auto reset_state = [&](RowState& rs) {   // all threads; the copy must be idle
+  auto reset_state = [&]() {   // all threads; nobody may be reading the selection scratch
     if (tid == 0) {
       rs.n_cand = 0;
       rs.n_member = 0;
@@ -827,6 +855,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
       rs.max_key = 0;
     }
     if (tid < kHistBins) rs.hist[tid] = 0;
+  };
+
+  // Thread 0: leaves position g to the dense routines.
+  auto defer = [&](size_t g) {
+    const unsigned at = atomicAdd(a.dev_status + kFailCount, 1u);
+    a.fail_list[at] = (int32_t)g;
+    atomicAdd(a.dev_status + kCntRows, 1u);
   };
 
   // One thread: the uniforms of a target position and the logit of x~ there.
@@ -868,161 +903,155 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
       }
       float pivot, inv_w;
       choose_pivot(0, std::false_type{}, pivot, inv_w);
-      stream_row(std::true_type{}, std::false_type{}, pivot, inv_w, true);
-      RowState& rs = sm.rs[rowi & 1];
+      stream_row(std::true_type{}, std::false_type{}, pivot, inv_w);
       __syncthreads();
-      reset_state(sm.rs[(rowi + 1) & 1]);
       Sel s;
-      bool ok = locate_bin(rs, s);
+      bool ok = locate_bin(s);
       float theta = 0.f;
       int n_ge = 0;
       double Zq = 1.0;
-      if (ok) exp_pass(std::true_type{}, rs, s, pivot, inv_w);
+      if (ok) exp_pass(std::true_type{}, s, pivot, inv_w);
       __syncthreads();
-      if (ok) ok = finish_selection(std::true_type{}, rs, s, theta, n_ge, Zq);
+      if (ok) ok = finish_selection(std::true_type{}, s, theta, n_ge, Zq);
       if (tid == 0) {
         learn(0, ok, theta, pivot, s.n, n_ge);
         sm.q_ok = ok;
         if (ok) {
+          // same rounding of Z_q as the unfused path (fp32 hi + lo)
+          const float Zhi = (float)Zq, Zlo = (float)(Zq - (double)Zhi);
+          const double Z = (double)Zhi + (double)Zlo;
+          RowSrc qr = {a.draft + (size_t)parent * P.V * esz, nullptr, 0.f, P.invT, P.V, BF16};
+          const float zq_tok = load1(qr, sm.tok);
+          const double q = (zq_tok >= theta) ? exp((double)zq_tok - (double)s.m) / Z : 0.0;
+          if (q <= 0.0) atomicOr(a.dev_status, MULO_DEV_ZERO_DRAFT_PROB);
           sm.theta_q = theta;
           sm.m_q = s.m;
-          sm.Zq = Zq;
+          sm.Zq = Z;
+          sm.q_tok = q;
+          sm.invZq = (float)(1.0 / Z);
         } else {
           atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
-          atomicAdd(a.dev_status + kCntRows, 1u);
+          for (int child = 0; child < rr; ++child)
+            defer((size_t)sm.b * P.H * P.W + (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r);
         }
       }
-      if (!ok) {   // block-uniform
-        __syncthreads();
-        dense_fallback_stats(a, sm, parent, bs);
-      }
-      __syncthreads();
-      if (tid == 0) {
-        // same rounding of Z_q as the unfused path (fp32 hi + lo)
-        const float Zhi = (float)sm.Zq, Zlo = (float)(sm.Zq - (double)Zhi);
-        const double Z = (double)Zhi + (double)Zlo;
-        RowSrc qr = {a.draft + (size_t)parent * P.V * esz, nullptr, 0.f, P.invT, P.V, BF16};
-        const float zq_tok = load1(qr, sm.tok);
-        const double q = (zq_tok >= sm.theta_q) ? exp((double)zq_tok - (double)sm.m_q) / Z : 0.0;
-        if (q <= 0.0) atomicOr(a.dev_status, MULO_DEV_ZERO_DRAFT_PROB);
-        sm.Zq = Z;
-        sm.q_tok = q;
-        sm.invZq = (float)(1.0 / Z);
-      }
-      if (tid == 64) prepare_row(sm.prep[(rowi + 1) & 1], 0);   // first child's uniforms and logit of x~
-      ++rowi;
+      __syncthreads();   // everybody is done with the selection scratch
+      reset_state();
+      if (tid == 64 && ok) prepare_row(sm.prep[rowi & 1], 0);   // first child's uniforms and logit of x~
       __syncthreads();
     }
 
     // ------------------------------------------------------------ children
-    for (int child = 0; child < P.r * P.r; ++child) {
-      const bool q_ok = sm.q_ok != 0;
-      RowState& rs = sm.rs[rowi & 1];
-      const RowPrep& pp = sm.prep[rowi & 1];
-      float pivot, inv_w;
-      choose_pivot(1, std::integral_constant<bool, HAS_U>{}, pivot, inv_w);
-      stream_row(std::false_type{}, std::integral_constant<bool, HAS_U>{}, pivot, inv_w, q_ok);
+    if (!sm.q_ok) {   // block-uniform: the whole parent went to the dense routines
+      for (int child = 0; child < rr; ++child) skip_row();
       __syncthreads();
-      reset_state(sm.rs[(rowi + 1) & 1]);
-      Sel s;
-      s.n = 0;
-      s.m = 0.f;
-      bool ok = q_ok && locate_bin(rs, s);
-      if (ok) {
-        if (tid == 32) sm.e_tok = exp((double)pp.z_tok - (double)s.m);
-        exp_pass(std::false_type{}, rs, s, pivot, inv_w);
-      }
-      __syncthreads();
-      float theta = 0.f;
-      int n_ge = 0;
-      double Zp = 1.0;
-      if (ok) ok = finish_selection(std::false_type{}, rs, s, theta, n_ge, Zp);
-      if (tid == 0 && q_ok) learn(1, ok, theta, pivot, s.n, n_ge);
-      const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
-      const size_t g = (size_t)sm.b * P.H * P.W + t;
-
-      if (ok) {
-        // ---- the decision (Eq. 1 / Eq. 5), the same in every warp
-        const double e_tok = (pp.z_tok >= theta) ? sm.e_tok : 0.0;
-        const double q_tok = sm.q_tok;
-        int accepted;
-        if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = e_tok >= P.tau * Zp;
-        else if (q_tok <= 0.0) accepted = e_tok > 0.0;
-        else accepted = uniform24(pp.rnd[0]) * q_tok * Zp < e_tok;
-        const int draws = draws_for(P.resample_mode, accepted);
-        const float invZp = (float)(1.0 / Zp), invZq = sm.invZq;
-        if (tid == 0) {
-          a.flags[g] = accepted ? 0 : 1;
-          if (a.p_tok) a.p_tok[g] = (float)(e_tok / Zp);
-          if (a.q_tok) a.q_tok[g] = (float)q_tok;
-          if (a.accept_prob) {
-            const double p = e_tok / Zp;
-            double thr;
-            if (P.accept_mode == MULO_ACCEPT_THRESHOLD) thr = p;
-            else if (q_tok <= 0.0) thr = p > 0.0 ? 1.0 : 0.0;
-            else thr = fmin(1.0, p / q_tok);
-            a.accept_prob[g] = (float)thr;
+    } else {
+      for (int child = 0; child < rr; ++child) {
+        const RowPrep& pp = sm.prep[rowi & 1];
+        float pivot, inv_w;
+        choose_pivot(1, std::integral_constant<bool, HAS_U>{}, pivot, inv_w);
+        stream_row(std::false_type{}, std::integral_constant<bool, HAS_U>{}, pivot, inv_w);
+        __syncthreads();
+        Sel s;
+        bool ok = locate_bin(s);
+        if (ok) {
+          if (tid == 32) sm.e_tok = exp((double)pp.z_tok - (double)s.m);
+          exp_pass(std::false_type{}, s, pivot, inv_w);
+        }
+        __syncthreads();
+        float theta = 0.f;
+        int n_ge = 0;
+        double Zp = 1.0;
+        if (ok) ok = finish_selection(std::false_type{}, s, theta, n_ge, Zp);
+        if (tid == 0) learn(1, ok, theta, pivot, s.n, n_ge);
+        const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
+        const size_t g = (size_t)sm.b * P.H * P.W + t;
+        int draws = 0;
+        float invZp = 0.f, invZq = 0.f;
+        if (ok) {
+          // ---- the decision (Eq. 1 / Eq. 5), the same in every warp
+          const double e_tok = (pp.z_tok >= theta) ? sm.e_tok : 0.0;
+          const double q_tok = sm.q_tok;
+          int accepted;
+          if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = e_tok >= P.tau * Zp;
+          else if (q_tok <= 0.0) accepted = e_tok > 0.0;
+          else accepted = uniform24(pp.rnd[0]) * q_tok * Zp < e_tok;
+          draws = draws_for(P.resample_mode, accepted);
+          invZp = (float)(1.0 / Zp);
+          invZq = sm.invZq;
+          if (tid == 0) {
+            a.flags[g] = accepted ? 0 : 1;
+            if (a.p_tok) a.p_tok[g] = (float)(e_tok / Zp);
+            if (a.q_tok) a.q_tok[g] = (float)q_tok;
+            if (a.accept_prob) {
+              const double p = e_tok / Zp;
+              double thr;
+              if (P.accept_mode == MULO_ACCEPT_THRESHOLD) thr = p;
+              else if (q_tok <= 0.0) thr = p > 0.0 ? 1.0 : 0.0;
+              else thr = fmin(1.0, p / q_tok);
+              a.accept_prob[g] = (float)thr;
+            }
           }
+        } else if (tid == 0) {
+          atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
+          defer(g);
         }
         // weight of candidate i in the residual of Eq. 2 (lambda = 1)
         auto w_resid = [&](int i) {
-          const uint2 en = cand[i];
-          const float pe = __fmul_rn(__uint_as_float(en.x), invZp);
-          const int id = (int)en.y;
+          const float pe = __fmul_rn(tz[i], invZp);
+          const int id = (int)tidl[i];
           const unsigned cell = qcell[id / EPL];
           const int j = id % EPL;
           float qe = 0.f;
           if ((cell >> j) & 1u) qe = qval[(id / PIECE) * a.cap + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
           return fmaxf(__fsub_rn(pe, __fmul_rn(qe, invZq)), 0.f);
         };
-        auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
+        auto w_target = [&](int i) { return tz[i]; };
         if (draws & kDrawResidual) {   // block-uniform
-          const int lane = MULO_LANE, warp = MULO_WARP, sub = lane & (kSegLanes - 1);
-          for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
-            const int c = c0 + lane / kSegLanes;
-            const int seg = c * kWarps + warp;
-            float acc = 0.f;
-            if (c < a.n_chunks) {
-              const int cn = min((int)tcnt[seg], a.cap);
-              for (int sl = sub; sl < cn; sl += kSegLanes) acc += w_resid(seg * a.cap + sl);
+          for (int c0 = 0; c0 < a.n_chunks; c0 += 2) {
+            const int segA = c0 * kChunkPieces + grp * kSWarps + warp, segB = segA + kChunkPieces;
+            const bool hasB = c0 + 1 < a.n_chunks;
+            const int cnA = min((int)tcnt[segA], a.cap);
+            const int cnB = hasB ? min((int)tcnt[segB], a.cap) : 0;
+            float accA = 0.f, accB = 0.f;
+            for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
+              if (sl < cnA) accA += w_resid(segA * a.cap + sl);
+              if (sl < cnB) accB += w_resid(segB * a.cap + sl);
             }
             __syncwarp();
-            acc = seg_lanes_sum(acc);
-            if (sub == 0 && c < a.n_chunks) seg_b[seg] = acc;
+            accA = seg_lanes_sum(accA);
+            accB = seg_lanes_sum(accB);
+            if (sub == 0) {
+              seg_b[segA] = accA;
+              if (hasB) seg_b[segB] = accB;
+            }
           }
         }
         __syncthreads();
-        const int warp = MULO_WARP;
-        if (warp == 0) {
-          int t_res = -1;
-          if (draws & kDrawResidual) {
-            int at = warp_draw(seg_b, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_resid);
-            if (at < 0)   // residual without mass: the target weights, same uniform
-              at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_target);
-            t_res = at >= 0 ? (int)cand[at].y : -1;
+        reset_state();
+        if (ok) {
+          if (warp == 0) {
+            int t_res = -1;
+            if (draws & kDrawResidual) {
+              int at = warp_draw(seg_b, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_resid);
+              if (at < 0)   // residual without mass: the target weights, same uniform
+                at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_target);
+              t_res = at >= 0 ? (int)tidl[at] : -1;
+            }
+            if (lane == 0) a.cand_res[g] = t_res;
+          } else if (warp == 1) {
+            int t_tgt = -1;
+            if (draws & kDrawTarget) {
+              const int at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[2]), w_target);
+              t_tgt = at >= 0 ? (int)tidl[at] : -1;
+            }
+            if (lane == 0) a.cand_tgt[g] = t_tgt;
           }
-          if (MULO_LANE == 0) a.cand_res[g] = t_res;
-        } else if (warp == 1) {
-          int t_tgt = -1;
-          if (draws & kDrawTarget) {
-            const int at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[2]), w_target);
-            t_tgt = at >= 0 ? (int)cand[at].y : -1;
-          }
-          if (MULO_LANE == 0) a.cand_tgt[g] = t_tgt;
-        } else if (tid == 64 && child + 1 < P.r * P.r) {
-          prepare_row(sm.prep[(rowi + 1) & 1], child + 1);
         }
-      } else {
-        if (tid == 0) {
-          atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
-          atomicAdd(a.dev_status + kCntRows, 1u);
-        }
-        if (tid == 64 && child + 1 < P.r * P.r) prepare_row(sm.prep[(rowi + 1) & 1], child + 1);
+        if (tid == 64 && child + 1 < rr) prepare_row(sm.prep[(rowi + 1) & 1], child + 1);
+        ++rowi;
         __syncthreads();
-        dense_fallback_position(a, sm, g, t, (uint32_t)sm.b + P.image_offset, parent, bs);
       }
-      ++rowi;
-      __syncthreads();
     }
     // next parent's coordinates (made visible by the barriers of its draft row)
     if (tid == 0) {
@@ -1035,8 +1064,6 @@ __global__ void __launch_bounds__(kThreads, 2) k_round_stream(const __grid_const
       }
     }
   }
-#undef MULO_LANE
-#undef MULO_WARP
 }
 
 }  // namespace mulo
