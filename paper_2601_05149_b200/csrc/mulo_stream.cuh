@@ -199,9 +199,18 @@ struct RowPrep {    // per target row, prepared while the previous row is finish
   float z_tok;      // pre-processed target logit of x~
 };
 
+// Cursor of the next chunk to request into a ring slot: chunk within the row, row within
+// the parent, table slot of the parent.  One per ring slot, in shared memory; only the warp
+// that is last out of the slot touches it, and two uses of a slot are ordered by the slot's
+// own barrier.
+struct Cursor {
+  int left;          // chunks still to request into this slot
+  unsigned pos;      // c | j << 8 | table slot << 16
+};
 struct StreamSmem {
   uint64_t full[kStages];
   unsigned done[kStages];
+  Cursor cursor[kStages];
   RowState rs;
   RowPrep prep[2];
   Predictor pred[2];   // 0: draft rows, 1: target rows
@@ -217,15 +226,7 @@ struct StreamSmem {
   unsigned long long row_off[kTableParents][kMaxRowsPerParent];   // byte offsets of the rows within their tensors
 };
 
-// Cursor of the next chunk to request: chunk within the row, row within the parent,
-// table slot of the parent.  Every thread carries the same copy and advances it once
-// per consumed chunk, so whichever warp is last out of a ring slot can issue.
-struct Cursor {
-  int left;          // chunks still to request
-  unsigned pos;      // c | j << 8 | table slot << 16
-};
 __device__ __forceinline__ void cursor_advance(Cursor& w, int n_chunks, int rows_per_parent) {
-  --w.left;
   unsigned c = (w.pos & 0xffu) + 1u, j = (w.pos >> 8) & 0xffu, s = w.pos >> 16;
   if (c == (unsigned)n_chunks) {
     c = 0;
@@ -467,12 +468,19 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
   if (tid < kHistBins) rs.hist[tid] = 0;
   __syncthreads();
 
-  Cursor cur;
-  cur.pos = 0;
-  cur.left = (p_end - p_begin) * rows_per_parent * a.n_chunks;
-  for (int s = 0; s < kStages && cur.left > 0; ++s) {
-    if (tid == 0) cursor_issue<BF16, HAS_U>(cur, a, sm, ring, s);
-    cursor_advance(cur, a.n_chunks, rows_per_parent);
+  if (tid == 0) {   // the first chunks, and each slot's cursor kStages chunks further on
+    const int total = (p_end - p_begin) * rows_per_parent * a.n_chunks;
+    Cursor cur;
+    cur.pos = 0;
+    cur.left = 0;
+    for (int s = 0; s < kStages; ++s) {
+      if (s < total) cursor_issue<BF16, HAS_U>(cur, a, sm, ring, s);
+      Cursor nxt = cur;
+      for (int k = 0; k < kStages; ++k) cursor_advance(nxt, a.n_chunks, rows_per_parent);
+      nxt.left = total > s + kStages ? (total - s - 1) / kStages : 0;
+      sm.cursor[s] = nxt;
+      cursor_advance(cur, a.n_chunks, rows_per_parent);
+    }
   }
   int rslot = 0;          // ring slot of the next chunk to read
   uint32_t rphase = 0;    // and its phase
@@ -487,10 +495,16 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
       if (old == (unsigned)kSWarps - 1u) {
         sm.done[rslot] = 0;
         __threadfence_block();
-        if (cur.left > 0) cursor_issue<BF16, HAS_U>(cur, a, sm, ring, rslot);
+        Cursor cur = sm.cursor[rslot];
+        if (cur.left > 0) {
+          cursor_issue<BF16, HAS_U>(cur, a, sm, ring, rslot);
+          --cur.left;
+#pragma unroll
+          for (int k = 0; k < kStages; ++k) cursor_advance(cur, a.n_chunks, rows_per_parent);
+          sm.cursor[rslot] = cur;
+        }
       }
     }
-    if (cur.left > 0) cursor_advance(cur, a.n_chunks, rows_per_parent);
     if (++rslot == kStages) {
       rslot = 0;
       rphase ^= 1u;
@@ -584,7 +598,8 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
         if (c * a.chunk + e < P.V) {
           raw_mix<BF16, ROW_U>(rc[i], ru[i], P.cfg_scale, P.invT, z[i]);
 #pragma unroll
-          for (int j = 0; j < EPL; ++j) mask[i] |= (z[i][j] >= pivot ? 1u : 0u) << j;
+          for (int j = 0; j < EPL; ++j)
+            if (z[i][j] >= pivot) mask[i] |= 1u << j;
         }
       }
       int cnt[kPPW], inc[kPPW];
