@@ -634,16 +634,6 @@ static double inv_norm_cdf(double p) {
   return 0.5 * (lo + hi);
 }
 
-// P(X > c) for X ~ binomial(n, p)
-static double binom_tail(int n, double p, int c) {
-  double pmf = pow(1.0 - p, n), cdf = 0.0;
-  for (int x = 0; x <= c && x <= n; ++x) {
-    cdf += pmf;
-    pmf *= (double)(n - x) / (x + 1) * p / (1.0 - p);
-  }
-  return fmax(0.0, 1.0 - cdf);
-}
-
 // Fills `s` and returns the dynamic shared memory the streaming kernel needs, or 0 if these
 // parameters are not eligible (then the general kernel runs).
 static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s) {
@@ -661,18 +651,13 @@ static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s
   s->n_chunks = (V + s->chunk - 1) / s->chunk;
   if (s->n_chunks > 255) return 0;
   s->n_seg = s->n_chunks * kChunkPieces;
-  // capacity of a segment's list: the smallest multiple of 8 that a binomial(piece, density)
-  // count exceeds, in any of a row's segments, with probability <= 1e-4 at the steady-state
-  // density and <= 2e-2 at the bootstrap density
-  int cap = 8;
-  for (; cap < piece; cap += 8)
-    if (s->n_seg * binom_tail(piece, (double)(k + margin) / V, cap) <= 1e-4 &&
-        s->n_seg * binom_tail(piece, (double)(k + margin_boot) / V, cap) <= 2e-2)
-      break;
-  if (cap > piece) cap = piece;
-  if (cap > 248) return 0;
+  // capacity of a row's candidate array: the bootstrap density's mean plus six standard
+  // deviations of a binomial(V, density) count, rounded up to a multiple of 64
+  const double pb = (double)(k + margin_boot) / V;
+  int cap = (int)ceil(V * pb + 6.0 * sqrt(V * pb * (1.0 - pb)));
+  cap = (cap + 63) / 64 * 64;
+  if (cap > 65535) return 0;
   s->cap = cap;
-  if ((size_t)s->n_seg * cap > 65535) return 0;
   s->margin = margin;
   s->a_theta = (float)inv_norm_cdf(1.0 - (double)k / V);
   s->a_boot = (float)inv_norm_cdf(1.0 - (double)(k + margin_boot) / V);

@@ -1,16 +1,19 @@
 // The fast path of the fused round for rows with top-k on (no pooling).
 //
-// A persistent CTA (256 threads, two per SM) owns a contiguous range of parent
+// A persistent CTA (256 threads, three per SM) owns a contiguous range of parent
 // (low-res) cells.  For each parent it streams the draft row and then its r*r
-// target rows ONCE through a shared-memory ring of 32 KB slots filled by bulk-async
-// copies (cp.async.bulk + mbarrier); the warp that releases a slot last requests
-// the next chunk into it, so there is no producer thread to wait for.  A chunk
-// iteration has a fixed latency of several hundred cycles (barrier wait, shared
-// loads, release), so every warp works on four independent 32-lane pieces of the
-// row per iteration and releases the slot as soon as its data are in registers.
+// target rows ONCE through a shared-memory ring filled by bulk-async copies
+// (cp.async.bulk + mbarrier); the warp that releases a slot last requests the next
+// chunk into it, so there is no producer thread to wait for.  A chunk iteration has
+// a fixed latency of several hundred cycles (barrier wait, shared loads, release),
+// so every warp works on two independent 32-lane pieces of the row per iteration
+// and releases the slot as soon as its data are in registers; the kernel is bound
+// by instruction issue and latency, which is why it is shaped for three resident
+// CTAs per SM (80 registers per thread, under 78 KB of shared memory).
 // The streaming pass keeps only the entries above a predicted pivot (k plus a
-// margin) and writes them, in ascending token id, into one fixed-capacity list per
-// piece of the row ("segment").  Everything else -- the exact k-th largest value,
+// margin) and appends them, in ascending token id, to the list of their piece of
+// the row ("segment"); a segment's list is a run of one array shared by the row,
+// claimed with one atomic add.  Everything else -- the exact k-th largest value,
 // softmax, acceptance, residual and the inverse-CDF draws -- works on those ~k
 // candidates in shared memory.  Each warp post-processes the segments it wrote,
 // eight lanes per segment, and values every warp needs (threshold, partition sum,
@@ -111,7 +114,7 @@ __device__ __forceinline__ float fast_exp(float z, float m) {
 // ------------------------------------------------------------ configuration
 constexpr int kSThreads = 256;       // threads per CTA of the streaming kernel
 constexpr int kSWarps = kSThreads / 32;
-constexpr int kPPW = 4;              // pieces per warp per chunk (independent work per iteration)
+constexpr int kPPW = 2;              // pieces per warp per chunk (independent work per iteration)
 constexpr int kChunkPieces = kSWarps * kPPW;
 constexpr int kStages = 2;           // ring slots
 constexpr int kHistBins = 256;       // selection histogram bins
@@ -144,12 +147,12 @@ struct StreamArgs {
   int n_chunks;     // chunks per row = ceil(V / chunk)
   int n_seg;        // segments per row = n_chunks * kChunkPieces; segment c * kChunkPieces + p is piece p of
                     // chunk c, handled by warp p % kSWarps
-  int cap;          // candidate capacity per segment (multiple of 8, < 256)
+  int cap;          // candidate capacity of a row (all segments together)
   int margin;       // extra candidates aimed for in steady state
   float a_theta;    // Phi^-1(1 - k/V)
   float a_boot;     // Phi^-1(1 - (k + bootstrap margin)/V)
   // byte offsets into dynamic shared memory (computed on the host)
-  uint32_t slot_bytes, off_tz, off_tid, off_qval, off_tcnt, off_qcnt, off_qcell, off_sega, off_segb, off_segc;
+  uint32_t slot_bytes, off_cand, off_qval, off_tseg, off_qseg, off_qcell, off_sega, off_segb, off_segc;
 };
 
 inline size_t stream_align(size_t x) { return (x + 127) / 128 * 128; }
@@ -163,14 +166,12 @@ inline size_t stream_layout(StreamArgs& a, int esz) {
     off += stream_align(bytes);
     return (uint32_t)o;
   };
-  const size_t n_list = (size_t)a.n_seg * a.cap;
   a.slot_bytes = (uint32_t)((size_t)a.chunk * esz * 2);   // cond + uncond halves
   take((size_t)a.slot_bytes * kStages);                   // the ring sits at offset 0
-  a.off_tz = take(n_list * 4);      // float z, later e = exp(z - m), of the target row's candidates
-  a.off_tid = take(n_list * 2);     // uint16 their token ids
-  a.off_qval = take(n_list * 4);    // float z, later exp(z - m_q), of the draft row
-  a.off_tcnt = take((size_t)a.n_seg * 2);   // uint16 entries per segment, target row
-  a.off_qcnt = take((size_t)a.n_seg * 2);   // uint16 entries per segment, draft row
+  a.off_cand = take((size_t)a.cap * 8);   // uint2 (z, later e = exp(z - m); token id) of the target row's candidates
+  a.off_qval = take((size_t)a.cap * 4);   // float z, later exp(z - m_q), of the draft row's candidates
+  a.off_tseg = take((size_t)a.n_seg * 4); // ushort2 (first entry, entries) per segment, target row
+  a.off_qseg = take((size_t)a.n_seg * 4); // the same for the draft row
   a.off_qcell = take((size_t)a.n_chunks * a.chunk / epl * 2);   // uint16 per lane visit of the draft row:
                                                                 // survivor mask | (first slot << 8)
   a.off_sega = take((size_t)a.n_seg * 4);   // float per-segment sums of e without the threshold bin's entries
@@ -192,6 +193,7 @@ struct RowState {   // selection scratch of the row in work
   unsigned short member_at[kMemberCap];
   unsigned short member_seg[kMemberCap];
   unsigned n_cand, n_member, overflow, max_key;
+  unsigned alloc;   // entries of the row's candidate array handed out so far
 };
 
 struct RowPrep {    // per target row, prepared while the previous row is finished
@@ -347,13 +349,12 @@ __device__ __forceinline__ int warp_locate(int cnt, float y, W wfun) {
 }
 
 // One inverse-CDF draw over per-segment weight sums `seg` (segments in ascending
-// token id, entries in ascending id inside a segment): scans the segment sums in
-// double, finds the segment that holds u * total, then the entry inside it.
-// Returns the index into the candidate array, or -1 when the total is zero.
-// Call from all lanes of ONE warp.
+// token id, entries in ascending id inside a segment; `run[s]` = first entry and
+// number of entries of segment s): scans the segment sums in double, finds the
+// segment that holds u * total, then the entry inside it.  Returns the index into
+// the candidate array, or -1 when the total is zero.  Call from all lanes of ONE warp.
 template <class W>
-__device__ __forceinline__ int warp_draw(const float* seg, int n_seg, int cap, const uint16_t* cnt, double u,
-                                         W wfun) {
+__device__ __forceinline__ int warp_draw(const float* seg, int n_seg, const ushort2* run, double u, W wfun) {
   const int lane = threadIdx.x & 31;
   double total = 0.0;
   for (int s = lane; s < n_seg; s += 32) total += (double)seg[s];
@@ -374,11 +375,10 @@ __device__ __forceinline__ int warp_draw(const float* seg, int n_seg, int cap, c
     const unsigned hit = __ballot_sync(kFull, w > 0.0 && carry + inc > y);
     if (hit) {
       const int l = __ffs(hit) - 1;
-      const int sseg = base + l;
+      const ushort2 r = run[base + l];
       const double before = carry + __shfl_sync(kFull, inc - w, l);
-      const int at = warp_locate(min((int)cnt[sseg], cap), (float)(y - before),
-                                 [&](int i) { return wfun(sseg * cap + i); });
-      if (at >= 0) return sseg * cap + at;
+      const int at = warp_locate((int)r.y, (float)(y - before), [&](int i) { return wfun((int)r.x + i); });
+      if (at >= 0) return (int)r.x + at;
     }
     const unsigned pos = __ballot_sync(kFull, w > 0.0);
     if (pos) last_seg = base + 31 - __clz(pos);
@@ -386,8 +386,9 @@ __device__ __forceinline__ int warp_draw(const float* seg, int n_seg, int cap, c
   }
   if (last_seg < 0) return -1;
   // rounding left u * total at (or past) the end: the last entry with weight
-  const int at = warp_locate(min((int)cnt[last_seg], cap), 3.0e38f, [&](int i) { return wfun(last_seg * cap + i); });
-  return at >= 0 ? last_seg * cap + at : -1;
+  const ushort2 r = run[last_seg];
+  const int at = warp_locate((int)r.y, 3.0e38f, [&](int i) { return wfun((int)r.x + i); });
+  return at >= 0 ? (int)r.x + at : -1;
 }
 
 // where the k-th largest value lies in a row's selection histogram
@@ -400,7 +401,7 @@ struct Sel {
 };
 
 template <bool BF16, bool HAS_U>
-__global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_constant__ StreamArgs a) {
+__global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_constant__ StreamArgs a) {
   constexpr int EPL = BF16 ? 8 : 4;        // entries per lane visit (16 bytes of the conditional row)
   constexpr int PIECE = 32 * EPL;          // entries per warp visit = one segment
   constexpr int esz = BF16 ? 2 : 4;
@@ -410,11 +411,10 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane & (kSegLanes - 1), grp = lane / kSegLanes;
   unsigned char* const ring = dyn;
-  float* const tz = reinterpret_cast<float*>(dyn + a.off_tz);
-  uint16_t* const tidl = reinterpret_cast<uint16_t*>(dyn + a.off_tid);
+  uint2* const cand = reinterpret_cast<uint2*>(dyn + a.off_cand);
   float* const qval = reinterpret_cast<float*>(dyn + a.off_qval);
-  uint16_t* const tcnt = reinterpret_cast<uint16_t*>(dyn + a.off_tcnt);
-  uint16_t* const qcnt = reinterpret_cast<uint16_t*>(dyn + a.off_qcnt);
+  ushort2* const tseg = reinterpret_cast<ushort2*>(dyn + a.off_tseg);
+  ushort2* const qseg = reinterpret_cast<ushort2*>(dyn + a.off_qseg);
   uint16_t* const qcell = reinterpret_cast<uint16_t*>(dyn + a.off_qcell);
   float* const seg_a = reinterpret_cast<float*>(dyn + a.off_sega);
   float* const seg_b = reinterpret_cast<float*>(dyn + a.off_segb);
@@ -437,6 +437,7 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
     rs.n_member = 0;
     rs.overflow = 0;
     rs.max_key = 0;
+    rs.alloc = 0;
     for (int s = 0; s < 2; ++s) {
       sm.pred[s].have = 0;
       sm.pred[s].theta = 0.f;
@@ -571,14 +572,13 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
     }
   };
 
-  // Streams one row through the ring: entries with z >= pivot go, in ascending
-  // token id, to the fixed-capacity list of their segment.  Then (pass A) each
-  // warp histograms the low end of the lists it wrote and contributes to the
-  // row's maximum and candidate count.
+  // Streams one row through the ring: entries with z >= pivot are appended, in ascending
+  // token id, to the list of their segment.  Then (pass A) each warp histograms the low end
+  // of the lists it wrote and contributes to the row's maximum and candidate count.
   auto stream_row = [&](auto is_q_tag, auto has_u_tag, float pivot, float inv_w) {
     constexpr bool IS_Q = decltype(is_q_tag)::value;
     constexpr bool ROW_U = decltype(has_u_tag)::value;
-    uint16_t* const cnt_arr = IS_Q ? qcnt : tcnt;
+    ushort2* const run = IS_Q ? qseg : tseg;
     for (int c = 0; c < a.n_chunks; ++c) {
       mbar_wait(&sm.full[rslot], rphase, a.dev_status);
       const unsigned char* slot = ring + (size_t)rslot * a.slot_bytes;
@@ -613,60 +613,65 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
           if (lane >= o) inc[i] += t;
         }
       }
+      // lane 31 knows the segment's size: it claims a run of the row's array
+      int base[kPPW];
+#pragma unroll
+      for (int i = 0; i < kPPW; ++i) {
+        base[i] = 0;
+        if (lane == 31) {
+          base[i] = (int)atomicAdd(&rs.alloc, (unsigned)inc[i]);
+          const int seg = c * kChunkPieces + i * kSWarps + warp;
+          const bool fits = base[i] + inc[i] <= a.cap;
+          run[seg] = make_ushort2((unsigned short)(fits ? base[i] : 0), (unsigned short)(fits ? inc[i] : 0));
+          if (!fits) {
+            rs.overflow = 1;
+            base[i] = -1;
+          }
+        }
+      }
 #pragma unroll
       for (int i = 0; i < kPPW; ++i) {
         const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
         const int id0 = c * a.chunk + e;
-        const int seg = c * kChunkPieces + i * kSWarps + warp;
-        const int total = __shfl_sync(kFull, inc[i], 31);
+        const int b0 = __shfl_sync(kFull, base[i], 31);
         const int off = inc[i] - cnt[i];
-        if (lane == 31) cnt_arr[seg] = (uint16_t)total;
         if (IS_Q && id0 < P.V) qcell[id0 / EPL] = (uint16_t)(mask[i] | ((unsigned)min(off, 255) << 8));
-        if (total <= a.cap) {
+        if (b0 >= 0) {
           if (IS_Q) {
-            float* dst = qval + seg * a.cap + off;
+            float* dst = qval + b0 + off;
 #pragma unroll
             for (int j = 0; j < EPL; ++j)
               if ((mask[i] >> j) & 1u) *dst++ = z[i][j];
           } else {
-            float* dz = tz + seg * a.cap + off;
-            uint16_t* di = tidl + seg * a.cap + off;
+            uint2* dst = cand + b0 + off;
 #pragma unroll
             for (int j = 0; j < EPL; ++j)
-              if ((mask[i] >> j) & 1u) {
-                *dz++ = z[i][j];
-                *di++ = (uint16_t)(id0 + j);
-              }
+              if ((mask[i] >> j) & 1u) *dst++ = make_uint2(__float_as_uint(z[i][j]), (unsigned)(id0 + j));
           }
-        } else if (lane == 0) {
-          rs.overflow = 1;
         }
       }
     }
-    // ---- pass A over the lists this warp wrote: group `grp` of 8 lanes takes piece grp of each chunk
+    // ---- pass A over the lists this warp wrote: group `grp` of 8 lanes takes the warp's two
+    //      pieces of chunk grp, grp + 4, ...
     __syncwarp();
-    float* const val = IS_Q ? qval : tz;
     float mx = -INFINITY;
     unsigned mine = 0;
-    for (int c0 = 0; c0 < a.n_chunks; c0 += 2) {
-      const int segA = c0 * kChunkPieces + grp * kSWarps + warp, segB = segA + kChunkPieces;
-      const int cnA = min((int)cnt_arr[segA], a.cap);
-      const int cnB = c0 + 1 < a.n_chunks ? min((int)cnt_arr[segB], a.cap) : 0;
+    for (int c = grp; c < a.n_chunks; c += kSegGroups) {
+      const ushort2 rA = run[c * kChunkPieces + warp], rB = run[c * kChunkPieces + kSWarps + warp];
+      const int cnA = rA.y, cnB = rB.y;
       if (sub == 0) mine += (unsigned)(cnA + cnB);
       for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
-        // (a full segment keeps entries of earlier rows, which may lie below the pivot: the row is
-        // redone anyway, but the index must stay inside the histogram)
         if (sl < cnA) {
-          const float zz = val[segA * a.cap + sl];
+          const float zz = IS_Q ? qval[rA.x + sl] : __uint_as_float(cand[rA.x + sl].x);
           mx = fmaxf(mx, zz);
           const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
-          if (fb >= 0.f && fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+          if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
         }
         if (sl < cnB) {
-          const float zz = val[segB * a.cap + sl];
+          const float zz = IS_Q ? qval[rB.x + sl] : __uint_as_float(cand[rB.x + sl].x);
           mx = fmaxf(mx, zz);
           const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
-          if (fb >= 0.f && fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+          if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
         }
       }
     }
@@ -740,11 +745,9 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
   // and are left out of the segment sums for now.
   auto exp_pass = [&](auto is_q_tag, const Sel& s, float pivot, float inv_w) {
     constexpr bool IS_Q = decltype(is_q_tag)::value;
-    const uint16_t* cnt_arr = IS_Q ? qcnt : tcnt;
-    float* const val = IS_Q ? qval : tz;
-    auto one = [&](int seg, int sl, float& acc) {
-      const int at = seg * a.cap + sl;
-      const float z = val[at];
+    const ushort2* run = IS_Q ? qseg : tseg;
+    auto one = [&](int seg, int at, float& acc) {
+      const float z = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
       const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
       const int bin = fb < (float)kHistBins ? (int)fb : kHistBins;
       float e = 0.f;
@@ -759,27 +762,30 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
       } else {
         acc += e;
       }
-      val[at] = e;
+      if (IS_Q) qval[at] = e;
+      else cand[at].x = __float_as_uint(e);
     };
-    for (int c0 = 0; c0 < a.n_chunks; c0 += 2) {
-      const int segA = c0 * kChunkPieces + grp * kSWarps + warp, segB = segA + kChunkPieces;
-      const bool hasB = c0 + 1 < a.n_chunks;
-      const int cnA = min((int)cnt_arr[segA], a.cap);
-      const int cnB = hasB ? min((int)cnt_arr[segB], a.cap) : 0;
+    for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
+      const int c = c0 + grp;
+      const int segA = c * kChunkPieces + warp, segB = segA + kSWarps;
       float accA = 0.f, accB = 0.f;
-      for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
-        if (sl < cnA) one(segA, sl, accA);
-        if (sl < cnB) one(segB, sl, accB);
+      if (c < a.n_chunks) {
+        const ushort2 rA = run[segA], rB = run[segB];
+        const int cnA = rA.y, cnB = rB.y;
+        for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
+          if (sl < cnA) one(segA, rA.x + sl, accA);
+          if (sl < cnB) one(segB, rB.x + sl, accB);
+        }
       }
       __syncwarp();
       accA = seg_lanes_sum(accA);
       accB = seg_lanes_sum(accB);
-      if (sub == 0) {
+      if (sub == 0 && c < a.n_chunks) {
         seg_a[segA] = accA;
-        if (!IS_Q) seg_c[segA] = accA;
-        if (hasB) {
-          seg_a[segB] = accB;
-          if (!IS_Q) seg_c[segB] = accB;
+        seg_a[segB] = accB;
+        if (!IS_Q) {
+          seg_c[segA] = accA;
+          seg_c[segB] = accB;
         }
       }
     }
@@ -791,7 +797,6 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
   // below theta gets e = 0, one at or above it is added to the complete segment sum.
   auto finish_selection = [&](auto is_q_tag, const Sel& s, float& theta, int& n_ge, double& Z) -> bool {
     constexpr bool IS_Q = decltype(is_q_tag)::value;
-    float* const val = IS_Q ? qval : tz;
     const int mcount = (int)rs.n_member;   // <= kMemberCap: locate_bin checked the bin's size
     float th = 0.f;
     int less_at = 0;
@@ -822,11 +827,12 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
       const bool keep = rs.member_z[i] >= th;
       const bool own = (seg & (kSWarps - 1)) == warp;   // one of this warp's segments
       if (keep) {
-        const float e = val[at];
+        const float e = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
         z += (double)e;
         if (own && !IS_Q) atomicAdd(&seg_c[seg], e);
       } else if (own) {
-        val[at] = 0.f;
+        if (IS_Q) qval[at] = 0.f;
+        else cand[at].x = 0u;
       }
     }
     __syncwarp();
@@ -868,6 +874,7 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
       rs.n_member = 0;
       rs.overflow = 0;
       rs.max_key = 0;
+      rs.alloc = 0;
     }
     if (tid < kHistBins) rs.hist[tid] = 0;
   };
@@ -1013,32 +1020,35 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
         }
         // weight of candidate i in the residual of Eq. 2 (lambda = 1)
         auto w_resid = [&](int i) {
-          const float pe = __fmul_rn(tz[i], invZp);
-          const int id = (int)tidl[i];
+          const uint2 en = cand[i];
+          const float pe = __fmul_rn(__uint_as_float(en.x), invZp);
+          const int id = (int)en.y;
           const unsigned cell = qcell[id / EPL];
           const int j = id % EPL;
           float qe = 0.f;
-          if ((cell >> j) & 1u) qe = qval[(id / PIECE) * a.cap + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
+          if ((cell >> j) & 1u) qe = qval[(int)qseg[id / PIECE].x + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
           return fmaxf(__fsub_rn(pe, __fmul_rn(qe, invZq)), 0.f);
         };
-        auto w_target = [&](int i) { return tz[i]; };
+        auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
         if (draws & kDrawResidual) {   // block-uniform
-          for (int c0 = 0; c0 < a.n_chunks; c0 += 2) {
-            const int segA = c0 * kChunkPieces + grp * kSWarps + warp, segB = segA + kChunkPieces;
-            const bool hasB = c0 + 1 < a.n_chunks;
-            const int cnA = min((int)tcnt[segA], a.cap);
-            const int cnB = hasB ? min((int)tcnt[segB], a.cap) : 0;
+          for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
+            const int c = c0 + grp;
+            const int segA = c * kChunkPieces + warp, segB = segA + kSWarps;
             float accA = 0.f, accB = 0.f;
-            for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
-              if (sl < cnA) accA += w_resid(segA * a.cap + sl);
-              if (sl < cnB) accB += w_resid(segB * a.cap + sl);
+            if (c < a.n_chunks) {
+              const ushort2 rA = tseg[segA], rB = tseg[segB];
+              const int cnA = rA.y, cnB = rB.y;
+              for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
+                if (sl < cnA) accA += w_resid(rA.x + sl);
+                if (sl < cnB) accB += w_resid(rB.x + sl);
+              }
             }
             __syncwarp();
             accA = seg_lanes_sum(accA);
             accB = seg_lanes_sum(accB);
-            if (sub == 0) {
+            if (sub == 0 && c < a.n_chunks) {
               seg_b[segA] = accA;
-              if (hasB) seg_b[segB] = accB;
+              seg_b[segB] = accB;
             }
           }
         }
@@ -1048,17 +1058,17 @@ __global__ void __launch_bounds__(kSThreads, 2) k_round_stream(const __grid_cons
           if (warp == 0) {
             int t_res = -1;
             if (draws & kDrawResidual) {
-              int at = warp_draw(seg_b, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_resid);
+              int at = warp_draw(seg_b, a.n_seg, tseg, uniform24(pp.rnd[1]), w_resid);
               if (at < 0)   // residual without mass: the target weights, same uniform
-                at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[1]), w_target);
-              t_res = at >= 0 ? (int)tidl[at] : -1;
+                at = warp_draw(seg_c, a.n_seg, tseg, uniform24(pp.rnd[1]), w_target);
+              t_res = at >= 0 ? (int)cand[at].y : -1;
             }
             if (lane == 0) a.cand_res[g] = t_res;
           } else if (warp == 1) {
             int t_tgt = -1;
             if (draws & kDrawTarget) {
-              const int at = warp_draw(seg_c, a.n_seg, a.cap, tcnt, uniform24(pp.rnd[2]), w_target);
-              t_tgt = at >= 0 ? (int)tidl[at] : -1;
+              const int at = warp_draw(seg_c, a.n_seg, tseg, uniform24(pp.rnd[2]), w_target);
+              t_tgt = at >= 0 ? (int)cand[at].y : -1;
             }
             if (lane == 0) a.cand_tgt[g] = t_tgt;
           }
