@@ -32,6 +32,29 @@ from paper_2601_05149_b200 import synth  # noqa: E402
 METRIC = "verified_grid_positions_per_sec"
 UNIT = "positions/s"
 
+# DRAM traffic of the streaming kernel per grid position (dram__bytes_read.sum + dram__bytes_write.sum of
+# one ncu capture of the C4 workload at B = 2, divided by its 8192 positions; traffic grows in proportion
+# to the positions, every row being read once).  None once the kernel has changed since the capture.
+TRAFFIC_BYTES_PER_POSITION = {"C4": None}
+
+
+def shard_for_rank(cfg, rank):
+    """Batch sharding over ranks: every rank runs cfg.B images of its own (weak scaling); the global image
+    indices of rank r are [r * B, (r + 1) * B), which is also what keys its random streams."""
+    return dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank), rank * cfg.B
+
+
+def reduce_max_ms(dist, elapsed_ms, device):
+    """The slowest rank's device time (all ranks get it)."""
+    t = torch.tensor([elapsed_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, positions_per_rank, steps, elapsed_ms):
+    """Positions per second of the whole job: what all ranks processed over the slowest rank's time."""
+    return world * positions_per_rank * steps / (elapsed_ms * 1e-3)
+
 
 def workload_desc(cfg):
     return (f"{cfg.name}: B={cfg.B} target {cfg.H}x{cfg.W} / draft {cfg.h}x{cfg.w}, V={cfg.V}, {cfg.dtype} "
@@ -180,9 +203,9 @@ def run_ours(args, cfg):
     dev = torch.device("cuda", local)
 
     # this rank's images: global indices [rank*B, (rank+1)*B)
-    rcfg = dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+    rcfg, image_offset = shard_for_rank(cfg, rank)
     batch = synth.build_batch(rcfg, dev)
-    p = binding.params_from_config(cfg, image_offset=rank * cfg.B)
+    p = binding.params_from_config(cfg, image_offset=image_offset)
     ctx.ensure_workspace(p)
     out = binding.alloc_round_outputs(p, dev, probs=False)
     stream = torch.cuda.current_stream()
@@ -222,13 +245,11 @@ def run_ours(args, cfg):
     ctx.set_timing(0)
     launches = ctx.kernel_launches() - launches0
     if dist:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+        elapsed_ms = reduce_max_ms(dist, elapsed_ms, dev)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
 
     positions = cfg.B * cfg.H * cfg.W
-    value = world * positions * K / (elapsed_ms * 1e-3)
+    value = whole_job_value(world, positions, K, elapsed_ms)
     n_rej = int(out["n_reject"].sum().item())
     n_exp = int(out["n_expand"].sum().item())
     status = ctx.poll_device_status()
@@ -247,12 +268,9 @@ def run_ours(args, cfg):
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                 "frac_of_nominal_8TBps": achieved / 8000.0, "traffic": None,
                 "bytes_per_launch": alg_bytes, "avg_launch_ms": row_avg_ms, "launches_timed": row_n}
-    tr = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tr):
-        try:
-            roofline["traffic"] = json.load(open(tr)).get(cfg.name)
-        except (ValueError, OSError):
-            pass
+    per_pos = TRAFFIC_BYTES_PER_POSITION.get(args.workload)
+    if per_pos is not None:
+        roofline["traffic"] = per_pos * positions
 
     e2e = None
     cpu = None
