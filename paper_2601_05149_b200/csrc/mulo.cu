@@ -655,6 +655,7 @@ static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s
   // deviations of a binomial(V, density) count, rounded up to a multiple of 64
   const double pb = (double)(k + margin_boot) / V;
   int cap = (int)ceil(V * pb + 6.0 * sqrt(V * pb * (1.0 - pb)));
+  cap += s->n_seg;              // every segment's run is rounded up to an even length
   cap = (cap + 63) / 64 * 64;
   if (cap > 65535) return 0;
   s->cap = cap;

@@ -602,41 +602,41 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
             if (z[i][j] >= pivot) mask[i] |= 1u << j;
         }
       }
-      int cnt[kPPW], inc[kPPW];
-#pragma unroll
-      for (int i = 0; i < kPPW; ++i) inc[i] = cnt[i] = __popc(mask[i]);
+      // one warp scan for both pieces' counts (16 bits each); lane 31 then claims one run of
+      // the row's array for the two segments, each rounded up to an even length so that the
+      // list passes can load entries in aligned pairs
+      static_assert(kPPW == 2, "the packed scan below handles two pieces");
+      const unsigned cnt0 = __popc(mask[0]), cnt1 = __popc(mask[1]);
+      unsigned inc = cnt0 | (cnt1 << 16);
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-#pragma unroll
-        for (int i = 0; i < kPPW; ++i) {
-          const int t = __shfl_up_sync(kFull, inc[i], o);
-          if (lane >= o) inc[i] += t;
+        const unsigned t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+      }
+      const unsigned tot = __shfl_sync(kFull, inc, 31);
+      const int t0 = (int)(tot & 0xffffu), t1 = (int)(tot >> 16);
+      const int t0e = (t0 + 1) & ~1, t1e = (t1 + 1) & ~1;
+      int base = 0;
+      if (lane == 31) {
+        base = (int)atomicAdd(&rs.alloc, (unsigned)(t0e + t1e));
+        const bool fits = base + t0e + t1e <= a.cap;
+        const int seg = c * kChunkPieces + warp;
+        run[seg] = make_ushort2((unsigned short)(fits ? base : 0), (unsigned short)(fits ? t0 : 0));
+        run[seg + kSWarps] = make_ushort2((unsigned short)(fits ? base + t0e : 0), (unsigned short)(fits ? t1 : 0));
+        if (!fits) {
+          rs.overflow = 1;
+          base = -1;
         }
       }
-      // lane 31 knows the segment's size: it claims a run of the row's array
-      int base[kPPW];
-#pragma unroll
-      for (int i = 0; i < kPPW; ++i) {
-        base[i] = 0;
-        if (lane == 31) {
-          base[i] = (int)atomicAdd(&rs.alloc, (unsigned)inc[i]);
-          const int seg = c * kChunkPieces + i * kSWarps + warp;
-          const bool fits = base[i] + inc[i] <= a.cap;
-          run[seg] = make_ushort2((unsigned short)(fits ? base[i] : 0), (unsigned short)(fits ? inc[i] : 0));
-          if (!fits) {
-            rs.overflow = 1;
-            base[i] = -1;
-          }
-        }
-      }
+      base = __shfl_sync(kFull, base, 31);
 #pragma unroll
       for (int i = 0; i < kPPW; ++i) {
         const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
         const int id0 = c * a.chunk + e;
-        const int b0 = __shfl_sync(kFull, base[i], 31);
-        const int off = inc[i] - cnt[i];
+        const int off = i == 0 ? (int)(inc & 0xffffu) - (int)cnt0 : (int)(inc >> 16) - (int)cnt1;
+        const int b0 = i == 0 ? base : base + t0e;
         if (IS_Q && id0 < P.V) qcell[id0 / EPL] = (uint16_t)(mask[i] | ((unsigned)min(off, 255) << 8));
-        if (b0 >= 0) {
+        if (base >= 0) {
           if (IS_Q) {
             float* dst = qval + b0 + off;
 #pragma unroll
@@ -652,26 +652,43 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       }
     }
     // ---- pass A over the lists this warp wrote: group `grp` of 8 lanes takes the warp's two
-    //      pieces of chunk grp, grp + 4, ...
+    //      pieces of chunk grp, grp + 4, ...; a lane loads two neighbouring entries at a time
     __syncwarp();
     float mx = -INFINITY;
     unsigned mine = 0;
+    auto tally = [&](float zz) {
+      mx = fmaxf(mx, zz);
+      const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
+      if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+    };
     for (int c = grp; c < a.n_chunks; c += kSegGroups) {
       const ushort2 rA = run[c * kChunkPieces + warp], rB = run[c * kChunkPieces + kSWarps + warp];
       const int cnA = rA.y, cnB = rB.y;
       if (sub == 0) mine += (unsigned)(cnA + cnB);
-      for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
+      for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
         if (sl < cnA) {
-          const float zz = IS_Q ? qval[rA.x + sl] : __uint_as_float(cand[rA.x + sl].x);
-          mx = fmaxf(mx, zz);
-          const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
-          if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+          float z0, z1;
+          if (IS_Q) {
+            const float2 v = *reinterpret_cast<const float2*>(qval + rA.x + sl);
+            z0 = v.x, z1 = v.y;
+          } else {
+            const uint4 v = *reinterpret_cast<const uint4*>(cand + rA.x + sl);
+            z0 = __uint_as_float(v.x), z1 = __uint_as_float(v.z);
+          }
+          tally(z0);
+          if (sl + 1 < cnA) tally(z1);
         }
         if (sl < cnB) {
-          const float zz = IS_Q ? qval[rB.x + sl] : __uint_as_float(cand[rB.x + sl].x);
-          mx = fmaxf(mx, zz);
-          const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
-          if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+          float z0, z1;
+          if (IS_Q) {
+            const float2 v = *reinterpret_cast<const float2*>(qval + rB.x + sl);
+            z0 = v.x, z1 = v.y;
+          } else {
+            const uint4 v = *reinterpret_cast<const uint4*>(cand + rB.x + sl);
+            z0 = __uint_as_float(v.x), z1 = __uint_as_float(v.z);
+          }
+          tally(z0);
+          if (sl + 1 < cnB) tally(z1);
         }
       }
     }
@@ -746,8 +763,8 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
   auto exp_pass = [&](auto is_q_tag, const Sel& s, float pivot, float inv_w) {
     constexpr bool IS_Q = decltype(is_q_tag)::value;
     const ushort2* run = IS_Q ? qseg : tseg;
-    auto one = [&](int seg, int at, float& acc) {
-      const float z = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
+    // e of one entry (value z at index `at`); the crossing bin's entries are set aside
+    auto one = [&](int seg, int at, float z, float& acc) -> float {
       const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
       const int bin = fb < (float)kHistBins ? (int)fb : kHistBins;
       float e = 0.f;
@@ -762,8 +779,23 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       } else {
         acc += e;
       }
-      if (IS_Q) qval[at] = e;
-      else cand[at].x = __float_as_uint(e);
+      return e;
+    };
+    // a lane's pair of neighbouring entries of a segment (the second one may lie past its end)
+    auto pair = [&](int seg, ushort2 r, int sl, float& acc) {
+      const int at = r.x + sl;
+      const bool two = sl + 1 < r.y;
+      if (IS_Q) {
+        float2 v = *reinterpret_cast<float2*>(qval + at);
+        v.x = one(seg, at, v.x, acc);
+        if (two) v.y = one(seg, at + 1, v.y, acc);
+        *reinterpret_cast<float2*>(qval + at) = v;
+      } else {
+        uint4 v = *reinterpret_cast<uint4*>(cand + at);
+        v.x = __float_as_uint(one(seg, at, __uint_as_float(v.x), acc));
+        if (two) v.z = __float_as_uint(one(seg, at + 1, __uint_as_float(v.z), acc));
+        *reinterpret_cast<uint4*>(cand + at) = v;
+      }
     };
     for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
       const int c = c0 + grp;
@@ -772,9 +804,9 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       if (c < a.n_chunks) {
         const ushort2 rA = run[segA], rB = run[segB];
         const int cnA = rA.y, cnB = rB.y;
-        for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
-          if (sl < cnA) one(segA, rA.x + sl, accA);
-          if (sl < cnB) one(segB, rB.x + sl, accB);
+        for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
+          if (sl < cnA) pair(segA, rA, sl, accA);
+          if (sl < cnB) pair(segB, rB, sl, accB);
         }
       }
       __syncwarp();
@@ -1019,15 +1051,24 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
           defer(g);
         }
         // weight of candidate i in the residual of Eq. 2 (lambda = 1)
-        auto w_resid = [&](int i) {
-          const uint2 en = cand[i];
-          const float pe = __fmul_rn(__uint_as_float(en.x), invZp);
-          const int id = (int)en.y;
+        auto w_entry = [&](unsigned ebits, unsigned idbits) {
+          const float pe = __fmul_rn(__uint_as_float(ebits), invZp);
+          const int id = (int)idbits;
           const unsigned cell = qcell[id / EPL];
           const int j = id % EPL;
           float qe = 0.f;
           if ((cell >> j) & 1u) qe = qval[(int)qseg[id / PIECE].x + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
           return fmaxf(__fsub_rn(pe, __fmul_rn(qe, invZq)), 0.f);
+        };
+        auto w_resid = [&](int i) {
+          const uint2 en = cand[i];
+          return w_entry(en.x, en.y);
+        };
+        auto w_pair = [&](ushort2 r, int sl) {
+          const uint4 v = *reinterpret_cast<const uint4*>(cand + r.x + sl);
+          float w = w_entry(v.x, v.y);
+          if (sl + 1 < r.y) w += w_entry(v.z, v.w);
+          return w;
         };
         auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
         if (draws & kDrawResidual) {   // block-uniform
@@ -1038,9 +1079,9 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
             if (c < a.n_chunks) {
               const ushort2 rA = tseg[segA], rB = tseg[segB];
               const int cnA = rA.y, cnB = rB.y;
-              for (int sl = sub; sl < max(cnA, cnB); sl += kSegLanes) {
-                if (sl < cnA) accA += w_resid(rA.x + sl);
-                if (sl < cnB) accB += w_resid(rB.x + sl);
+              for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
+                if (sl < cnA) accA += w_pair(rA, sl);
+                if (sl < cnB) accB += w_pair(rB, sl);
               }
             }
             __syncwarp();
