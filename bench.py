@@ -338,6 +338,67 @@ def run_e2e(ctx, cfg, p, batch, world, args):
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "n_gpus": 1}
 
 
+def run_sweep(args):
+    """The throughput sweep (grids x vocabularies x batches x noise levels): one JSON line per point with
+    positions/s, the HBM roofline fraction of the row kernels and the measured acceptance.  Single GPU."""
+    from paper_2601_05149_b200 import binding
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the round has no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    ctx = binding.Context(0)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else 6650.0
+    pts = synth.sweep_points()
+    if args.sweep_limit:
+        pts = pts[:args.sweep_limit]
+    groups = {}
+    for c in pts:
+        groups.setdefault((c.H, c.V, c.sigma), []).append(c)
+    K, Wm = max(1, min(args.steps, 5)), 3
+    for (g, V, sigma), cs in groups.items():
+        big = max(cs, key=lambda c: c.B)
+        batch = synth.build_batch(big, dev)      # the smaller batches are its leading images
+        for c in sorted(cs, key=lambda c: c.B):
+            cut = {k: (v if v is None or k == "nn" else v[:c.B]) for k, v in batch.items()}
+            p = binding.params_from_config(dataclasses.replace(big, B=c.B))
+            ctx.ensure_workspace(p)
+            out = binding.alloc_round_outputs(p, dev, probs=False)
+
+            def step(rnd):
+                p.round = rnd
+                ctx.mulo_round(p, cut["cond"], cut["uncond"], cut["draft_lo"], cut["tok_lo"], cut["nn"],
+                               out["out_tok"], out["reject_bits"], out["expand_bits"], None, None, None,
+                               out["n_reject"], out["n_expand"], out["first_reject"])
+            for s_ in range(Wm):
+                step(s_)
+            torch.cuda.synchronize()
+            ctx.set_timing(K)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for s_ in range(K):
+                step(Wm + s_)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / K
+            row_ms, row_n = ctx.read_timing()
+            ctx.set_timing(0)
+            positions = c.B * c.H * c.W
+            alg = c.algorithmic_bytes_per_position() * positions
+            gbs = alg / (row_ms / max(1, row_n) * 1e-3) / 1e9
+            print(json.dumps({
+                "sweep_point": c.name, "grid": c.H, "V": c.V, "B": c.B, "sigma": c.sigma, "metric": METRIC,
+                "value": positions / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+                "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak},
+                "l2_resident": alg < 126e6,
+                "acceptance_rate": 1.0 - int(out["n_reject"].sum().item()) / positions,
+                "expanded_fraction": int(out["n_expand"].sum().item()) / positions,
+                "rows_redone_by_general_kernel": ctx.poll_fallback_counts()[0]}), flush=True)
+        del batch
+        torch.cuda.empty_cache()
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -347,11 +408,15 @@ def main():
     ap.add_argument("--workload", default="C4", choices=sorted(synth.CONFIGS))
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the bench line")
+    ap.add_argument("--sweep-limit", type=int, default=0, help="only the first N sweep points")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.workload]
     if args.batch:
         cfg = dataclasses.replace(cfg, B=args.batch, name=f"{cfg.name}(B={args.batch})")
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_ours(args, cfg)

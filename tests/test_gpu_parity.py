@@ -300,3 +300,14 @@ def test_config_C4_sampled_images(ctx):
         else:   # only the masks and the choice of draw depend on the radius
             o = pu.oracle_images(c, batch, [cfg.B - 1])
         pu.check_round(c, g, o)
+
+
+@pytest.mark.parametrize("pick", [0, 43, 95], ids=["32x32-V8192-s0.1", "64x64-V8192-s2.0", "96x96-V16384-s2.0"])
+def test_sweep_points_sampled(ctx, pick):
+    """Points of the throughput sweep (batch cut to 2 images to bound the oracle's time)."""
+    cfg = dataclasses.replace(synth.sweep_points()[pick], B=2)
+    batch = pu.build_batch(cfg)
+    g = pu.gpu_round(ctx, cfg, batch)
+    assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
+    o = pu.oracle_images(cfg, batch, [1])
+    pu.check_round(cfg, g, o)
