@@ -356,39 +356,46 @@ __device__ __forceinline__ int warp_locate(int cnt, float y, W wfun) {
 template <class W>
 __device__ __forceinline__ int warp_draw(const float* seg, int n_seg, const ushort2* run, double u, W wfun) {
   const int lane = threadIdx.x & 31;
-  double total = 0.0;
-  for (int s = lane; s < n_seg; s += 32) total += (double)seg[s];
-  total = warp_sum(total);
+  // every lane sums a block of consecutive segments, then one scan over the lanes
+  const int per = (n_seg + 31) / 32;
+  const int s0 = lane * per;
+  double loc = 0.0;
+  for (int i = 0; i < per; ++i)
+    if (s0 + i < n_seg) loc += (double)seg[s0 + i];
+  double inc = loc;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const double t = __shfl_up_sync(kFull, inc, o);
+    if (lane >= o) inc += t;
+  }
+  const double total = __shfl_sync(kFull, inc, 31);
   if (!(total > 0.0)) return -1;
   const double y = u * total;
-  double carry = 0.0;
-  int last_seg = -1;
-  for (int base = 0; base < n_seg; base += 32) {
-    const int s = base + lane;
-    const double w = s < n_seg ? (double)seg[s] : 0.0;
-    double inc = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      double t = __shfl_up_sync(kFull, inc, o);
-      if (lane >= o) inc += t;
+  const unsigned hit = __ballot_sync(kFull, loc > 0.0 && inc > y);
+  if (hit) {
+    const int l = __ffs(hit) - 1;
+    double acc = __shfl_sync(kFull, inc - loc, l);   // mass before lane l's block
+    for (int i = 0; i < per; ++i) {                  // the same walk in every lane
+      const int sidx = l * per + i;
+      if (sidx >= n_seg) break;
+      const double w = (double)seg[sidx];
+      if (w > 0.0 && acc + w > y) {
+        const ushort2 r = run[sidx];
+        const int at = warp_locate((int)r.y, (float)(y - acc), [&](int k) { return wfun((int)r.x + k); });
+        if (at >= 0) return (int)r.x + at;
+      }
+      acc += w;
     }
-    const unsigned hit = __ballot_sync(kFull, w > 0.0 && carry + inc > y);
-    if (hit) {
-      const int l = __ffs(hit) - 1;
-      const ushort2 r = run[base + l];
-      const double before = carry + __shfl_sync(kFull, inc - w, l);
-      const int at = warp_locate((int)r.y, (float)(y - before), [&](int i) { return wfun((int)r.x + i); });
+  }
+  // rounding left u * total at (or past) the end: the last entry with weight
+  for (int sidx = n_seg - 1; sidx >= 0; --sidx) {
+    if (seg[sidx] > 0.f) {
+      const ushort2 r = run[sidx];
+      const int at = warp_locate((int)r.y, 3.0e38f, [&](int k) { return wfun((int)r.x + k); });
       if (at >= 0) return (int)r.x + at;
     }
-    const unsigned pos = __ballot_sync(kFull, w > 0.0);
-    if (pos) last_seg = base + 31 - __clz(pos);
-    carry += __shfl_sync(kFull, inc, 31);
   }
-  if (last_seg < 0) return -1;
-  // rounding left u * total at (or past) the end: the last entry with weight
-  const ushort2 r = run[last_seg];
-  const int at = warp_locate((int)r.y, 3.0e38f, [&](int i) { return wfun((int)r.x + i); });
-  return at >= 0 ? (int)r.x + at : -1;
+  return -1;
 }
 
 // where the k-th largest value lies in a row's selection histogram
@@ -420,6 +427,11 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
   float* const seg_b = reinterpret_cast<float*>(dyn + a.off_segb);
   float* const seg_c = reinterpret_cast<float*>(dyn + a.off_segc);
   RowState& rs = sm.rs;
+  // The 2 * n_chunks segments this warp writes, in ascending token id: number i is piece i % 2 of
+  // chunk i / 2.  In the list passes group `grp` of 8 lanes takes numbers grp and grp + 4 (then
+  // + 8, ...), two segments side by side for instruction-level parallelism.
+  const int nsw = kPPW * a.n_chunks;
+  auto seg_of = [&](int i) { return (i >> 1) * kChunkPieces + (i & 1) * kSWarps + warp; };
 
   // this CTA's parents: [p_begin, p_end)
   const int p_begin = (int)(((long long)a.n_parents * blockIdx.x) / gridDim.x);
@@ -661,8 +673,9 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
       if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
     };
-    for (int c = grp; c < a.n_chunks; c += kSegGroups) {
-      const ushort2 rA = run[c * kChunkPieces + warp], rB = run[c * kChunkPieces + kSWarps + warp];
+    for (int iA = grp; iA < nsw; iA += 2 * kSegGroups) {
+      const int iB = iA + kSegGroups;
+      const ushort2 rA = run[seg_of(iA)], rB = iB < nsw ? run[seg_of(iB)] : make_ushort2(0, 0);
       const int cnA = rA.y, cnB = rB.y;
       if (sub == 0) mine += (unsigned)(cnA + cnB);
       for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
@@ -797,12 +810,13 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         *reinterpret_cast<uint4*>(cand + at) = v;
       }
     };
-    for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
-      const int c = c0 + grp;
-      const int segA = c * kChunkPieces + warp, segB = segA + kSWarps;
+    for (int i0 = 0; i0 < nsw; i0 += 2 * kSegGroups) {
+      const int iA = i0 + grp, iB = iA + kSegGroups;
+      const bool hasA = iA < nsw, hasB = iB < nsw;
+      const int segA = seg_of(iA), segB = seg_of(iB);
       float accA = 0.f, accB = 0.f;
-      if (c < a.n_chunks) {
-        const ushort2 rA = run[segA], rB = run[segB];
+      if (hasA) {
+        const ushort2 rA = run[segA], rB = hasB ? run[segB] : make_ushort2(0, 0);
         const int cnA = rA.y, cnB = rB.y;
         for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
           if (sl < cnA) pair(segA, rA, sl, accA);
@@ -812,12 +826,14 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       __syncwarp();
       accA = seg_lanes_sum(accA);
       accB = seg_lanes_sum(accB);
-      if (sub == 0 && c < a.n_chunks) {
-        seg_a[segA] = accA;
-        seg_a[segB] = accB;
-        if (!IS_Q) {
-          seg_c[segA] = accA;
-          seg_c[segB] = accB;
+      if (sub == 0) {
+        if (hasA) {
+          seg_a[segA] = accA;
+          if (!IS_Q) seg_c[segA] = accA;
+        }
+        if (hasB) {
+          seg_a[segB] = accB;
+          if (!IS_Q) seg_c[segB] = accB;
         }
       }
     }
@@ -1072,12 +1088,13 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         };
         auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
         if (draws & kDrawResidual) {   // block-uniform
-          for (int c0 = 0; c0 < a.n_chunks; c0 += kSegGroups) {
-            const int c = c0 + grp;
-            const int segA = c * kChunkPieces + warp, segB = segA + kSWarps;
+          for (int i0 = 0; i0 < nsw; i0 += 2 * kSegGroups) {
+            const int iA = i0 + grp, iB = iA + kSegGroups;
+            const bool hasA = iA < nsw, hasB = iB < nsw;
+            const int segA = seg_of(iA), segB = seg_of(iB);
             float accA = 0.f, accB = 0.f;
-            if (c < a.n_chunks) {
-              const ushort2 rA = tseg[segA], rB = tseg[segB];
+            if (hasA) {
+              const ushort2 rA = tseg[segA], rB = hasB ? tseg[segB] : make_ushort2(0, 0);
               const int cnA = rA.y, cnB = rB.y;
               for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
                 if (sl < cnA) accA += w_pair(rA, sl);
@@ -1087,9 +1104,9 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
             __syncwarp();
             accA = seg_lanes_sum(accA);
             accB = seg_lanes_sum(accB);
-            if (sub == 0 && c < a.n_chunks) {
-              seg_b[segA] = accA;
-              seg_b[segB] = accB;
+            if (sub == 0) {
+              if (hasA) seg_b[segA] = accA;
+              if (hasB) seg_b[segB] = accB;
             }
           }
         }
