@@ -643,7 +643,7 @@ static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s
   // candidates aimed for beyond k: about six standard deviations of the count of entries
   // above a fixed value near the k-th largest
   const int margin = (int)fmax(64.0, 6.0 * sqrt((double)k));
-  const int margin_boot = 2 * margin;
+  const int margin_boot = margin + 3 * margin / 4;   // rows without a prediction: the pivot comes from one chunk's statistics
   if ((double)(k + margin_boot) > 0.5 * V) return 0;
   const int esz = d.bf16 ? 2 : 4;
   const int epl = 16 / esz, piece = 32 * epl;
