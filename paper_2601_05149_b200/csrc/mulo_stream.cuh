@@ -185,6 +185,12 @@ inline size_t stream_layout(StreamArgs& a, int esz) {
 struct Predictor {
   int have;
   float theta, rho;
+  // rows without a prediction take the pivot from the mean and spread of their first chunk,
+  // assuming a normal shape; when that start fails, `shift` (in units of the spread) moves the
+  // next start down (too few candidates) or up (too many): the step doubles while the
+  // failures point the same way and halves when they change direction
+  float shift, step;
+  int dir;
 };
 
 struct RowState {   // selection scratch of the row in work
@@ -405,6 +411,8 @@ struct Sel {
   int want;     // its 1-based rank inside that bin, from below
   int cum;      // entries in the bins below
   float m;      // row maximum
+  int reason;   // why the row left the fast path: 0 not at all, 1 list full, 2 too few candidates,
+                // 3 k-th largest above the histogram, 4 too many ties at the threshold
 };
 
 template <bool BF16, bool HAS_U>
@@ -454,6 +462,9 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       sm.pred[s].have = 0;
       sm.pred[s].theta = 0.f;
       sm.pred[s].rho = 1.f;
+      sm.pred[s].shift = 0.f;
+      sm.pred[s].step = 0.f;
+      sm.pred[s].dir = 0;
     }
     const int hw = P.h * P.w;
     sm.b = p_begin / hw;
@@ -571,7 +582,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     const float mean = (float)(S1 / elems);
     const float sd = sqrtf(fmaxf((float)(S2 / elems) - mean * mean, 1e-20f));
     const float d = fmaxf((a.a_theta - a.a_boot) * sd, 1e-20f);
-    pivot = mean + a.a_boot * sd;
+    pivot = mean + (a.a_boot + pr.shift) * sd;
     inv_w = (float)kHistBins / (3.0f * d);
   };
 
@@ -720,8 +731,10 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
   auto locate_bin = [&](Sel& s) -> bool {
     const int k = P.top_k;
     s.n = (int)rs.n_cand;
+    s.reason = 0;
     if (rs.overflow || s.n < k) {
       if (tid == 0) atomicAdd(a.dev_status + (rs.overflow ? kCntListFull : kCntTooFew), 1u);
+      s.reason = rs.overflow ? 1 : 2;
       return false;
     }
     s.m = key_float(rs.max_key);
@@ -743,6 +756,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     const unsigned owner_mask = __ballot_sync(kFull, inc >= (unsigned)rank);
     if (owner_mask == 0) {   // the rank lies above the histogram range
       if (tid == 0) atomicAdd(a.dev_status + kCntAboveRange, 1u);
+      s.reason = 3;
       return false;
     }
     const int owner = __ffs(owner_mask) - 1;
@@ -765,6 +779,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     s.want = rank - s.cum;
     if (in_bin > (unsigned)kMemberCap) {
       if (tid == 0) atomicAdd(a.dev_status + kCntCrowdedBin, 1u);
+      s.reason = 4;
       return false;
     }
     return true;
@@ -892,11 +907,21 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
   };
 
   // Thread 0: the predictor of a kind of row after a row (ok: theta found exactly).
-  auto learn = [&](int kind, bool ok, float theta, float pivot, int n, int n_ge) {
+  auto learn = [&](int kind, bool ok, int reason, float theta, float pivot, int n, int n_ge) {
     Predictor pr = sm.pred[kind];
     if (!ok) {
       pr.have = 0;
+      const int dir = reason == 2 ? -1 : (reason == 1 || reason == 3) ? 1 : 0;
+      if (dir != 0) {
+        const float unit = 0.5f * (a.a_theta - a.a_boot);
+        if (pr.dir == 0) pr.step = unit;
+        else if (pr.dir == dir) pr.step = fminf(2.0f * pr.step, 64.0f * unit);
+        else pr.step = fmaxf(0.5f * pr.step, 0.25f * unit);
+        pr.shift += (float)dir * pr.step;
+        pr.dir = dir;
+      }
     } else {
+      pr.dir = 0;
       const int below = n - n_ge;   // candidates in [pivot, theta)
       float rho = pr.rho;
       bool rho_ok = pr.have != 0;
@@ -984,7 +1009,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       __syncthreads();
       if (ok) ok = finish_selection(std::true_type{}, s, theta, n_ge, Zq);
       if (tid == 0) {
-        learn(0, ok, theta, pivot, s.n, n_ge);
+        learn(0, ok, s.reason, theta, pivot, s.n, n_ge);
         sm.q_ok = ok;
         if (ok) {
           // same rounding of Z_q as the unfused path (fp32 hi + lo)
@@ -1033,7 +1058,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         int n_ge = 0;
         double Zp = 1.0;
         if (ok) ok = finish_selection(std::false_type{}, s, theta, n_ge, Zp);
-        if (tid == 0) learn(1, ok, theta, pivot, s.n, n_ge);
+        if (tid == 0) learn(1, ok, s.reason, theta, pivot, s.n, n_ge);
         const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
         const size_t g = (size_t)sm.b * P.H * P.W + t;
         int draws = 0;

@@ -19,6 +19,7 @@ def ctx():
     assert torch.cuda.is_available()
     binding.lib()            # raises if the library was not built: no fallback
     c = binding.Context(0)
+    c.set_workspace(torch.empty(1 << 16, dtype=torch.uint8, device="cuda"))   # so that status polls work from the start
     yield c
     assert c.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
     c.close()
@@ -310,4 +311,25 @@ def test_sweep_points_sampled(ctx, pick):
     g = pu.gpu_round(ctx, cfg, batch)
     assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
     o = pu.oracle_images(cfg, batch, [1])
+    pu.check_round(cfg, g, o)
+
+
+def test_fast_path_adapts_to_rows_that_are_not_normal(ctx):
+    """Heavy-tailed logits (cubed normals) defeat the normal-shaped first guess of the pivot; the guess
+    must adapt within a few rows, the rows it loses go to the general routines, results stay exact."""
+    cfg = dataclasses.replace(BIG, V=4096, top_k=500, B=8, H=64, W=64, seed=240)
+    batch = pu.build_batch(cfg)
+    for k in ("cond", "uncond", "draft_lo"):
+        x = batch[k].float()
+        batch[k] = (x * x * x / 8.0).to(batch[k].dtype).contiguous()
+    # draft tokens must have draft probability > 0 under the new logits: take each row's maximum
+    batch["tok_lo"] = batch["draft_lo"].float().argmax(-1).to(torch.int32).contiguous()
+    ctx.poll_device_status()
+    ctx.poll_fallback_counts()
+    g = pu.gpu_round(ctx, cfg, batch)
+    assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
+    lost = ctx.poll_fallback_counts()[0]
+    rows = cfg.B * cfg.H * cfg.W
+    assert lost < 0.6 * rows, (lost, rows)      # every CTA loses its first few parents while it adapts
+    o = pu.oracle_images(cfg, batch, [0, cfg.B - 1])
     pu.check_round(cfg, g, o)
