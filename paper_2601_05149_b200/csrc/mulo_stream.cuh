@@ -1072,7 +1072,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
           else if (q_tok <= 0.0) accepted = e_tok > 0.0;
           else accepted = uniform24(pp.rnd[0]) * q_tok * Zp < e_tok;
           draws = draws_for(P.resample_mode, accepted);
-          invZp = (float)(1.0 / Zp);
+          invZp = 1.0f / (float)Zp;
           invZq = sm.invZq;
           if (tid == 0) {
             a.flags[g] = accepted ? 0 : 1;
