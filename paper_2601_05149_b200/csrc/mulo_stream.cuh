@@ -70,6 +70,7 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded waits: give up, flag, carry on
 
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status) {
+#pragma unroll 1
   for (uint32_t it = 0; it < kSpinLimit; ++it)
     if (mbar_try_wait(bar, parity)) return;
   atomicOr(dev_status, MULO_DEV_TIMEOUT);   // the data is then garbage, but nothing hangs
