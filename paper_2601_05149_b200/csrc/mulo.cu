@@ -650,12 +650,16 @@ static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s
   s->chunk = kChunkPieces * piece;
   s->n_chunks = (V + s->chunk - 1) / s->chunk;
   if (s->n_chunks > 255) return 0;
-  s->n_seg = s->n_chunks * kChunkPieces;
+  s->n_seg = s->n_chunks * kSWarps;
   // capacity of a row's candidate array: the bootstrap density's mean plus six standard
   // deviations of a binomial(V, density) count, rounded up to a multiple of 64
   const double pb = (double)(k + margin_boot) / V;
   int cap = (int)ceil(V * pb + 6.0 * sqrt(V * pb * (1.0 - pb)));
   cap += s->n_seg;              // every segment's run is rounded up to an even length
+  {   // a segment of the draft row may hold at most 255 candidates (8-bit offsets in its look-up table)
+    const double seg_mean = (double)kPPW * piece * pb;
+    if (seg_mean + 6.0 * sqrt(seg_mean * (1.0 - pb)) > 255.0) return 0;
+  }
   cap = (cap + 63) / 64 * 64;
   if (cap > 65535) return 0;
   s->cap = cap;

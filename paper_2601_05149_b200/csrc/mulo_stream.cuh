@@ -120,8 +120,6 @@ constexpr int kChunkPieces = kSWarps * kPPW;
 constexpr int kStages = 2;           // ring slots
 constexpr int kHistBins = 256;       // selection histogram bins
 constexpr int kMemberCap = 128;      // entries of the crossing bin ranked exactly
-constexpr int kSegLanes = 8;         // lanes that share one segment in the list passes
-constexpr int kSegGroups = 32 / kSegLanes;
 constexpr int kTableParents = 4;     // parents whose row addresses are kept
 constexpr int kMaxRowsPerParent = 17;   // draft row + r*r children, r <= 4
 // words of the device status block after the flag word: rows redone by the general
@@ -146,8 +144,8 @@ struct StreamArgs {
   int n_parents;
   int chunk;        // elements per ring slot half = kChunkPieces pieces
   int n_chunks;     // chunks per row = ceil(V / chunk)
-  int n_seg;        // segments per row = n_chunks * kChunkPieces; segment c * kChunkPieces + p is piece p of
-                    // chunk c, handled by warp p % kSWarps
+  int n_seg;        // segments per row = n_chunks * kSWarps; segment c * kSWarps + w is the part of chunk c
+                    // that warp w handles: kPPW adjacent 32-lane pieces, i.e. kPPW * 32 * (16 / esz) entries
   int cap;          // candidate capacity of a row (all segments together)
   int margin;       // extra candidates aimed for in steady state
   float a_theta;    // Phi^-1(1 - k/V)
@@ -322,10 +320,9 @@ __device__ __forceinline__ void raw_mix(const uint4& c, const uint4& u, float s,
   }
 }
 
-__device__ __forceinline__ float seg_lanes_sum(float v) {
-  v += __shfl_xor_sync(kFull, v, 1);
-  v += __shfl_xor_sync(kFull, v, 2);
-  v += __shfl_xor_sync(kFull, v, 4);
+// sum over the `lanes` (a power of two) neighbouring lanes that share a segment
+__device__ __forceinline__ float seg_lanes_sum(float v, int lanes) {
+  for (int o = 1; o < lanes; o <<= 1) v += __shfl_xor_sync(kFull, v, o);
   return v;
 }
 
@@ -419,13 +416,18 @@ struct Sel {
 template <bool BF16, bool HAS_U>
 __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_constant__ StreamArgs a) {
   constexpr int EPL = BF16 ? 8 : 4;        // entries per lane visit (16 bytes of the conditional row)
-  constexpr int PIECE = 32 * EPL;          // entries per warp visit = one segment
+  constexpr int PIECE = 32 * EPL;          // entries per 32-lane piece
+  constexpr int SEG = kPPW * PIECE;        // entries of the row that one segment covers
   constexpr int esz = BF16 ? 2 : 4;
   __shared__ StreamSmem sm;
   extern __shared__ __align__(128) unsigned char dyn[];
   const DevParams& P = a.P;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int sub = lane & (kSegLanes - 1), grp = lane / kSegLanes;
+  // In the list passes a warp's lanes split into up to four groups, one segment per group
+  // at a time (group g takes the warp's segment of chunk g, g + groups, ...).
+  const int groups = a.n_chunks >= 3 ? 4 : a.n_chunks;   // 1, 2 or 4
+  const int seg_lanes = 32 / groups;
+  const int sub = lane & (seg_lanes - 1), grp = lane / seg_lanes;
   unsigned char* const ring = dyn;
   uint2* const cand = reinterpret_cast<uint2*>(dyn + a.off_cand);
   float* const qval = reinterpret_cast<float*>(dyn + a.off_qval);
@@ -436,11 +438,6 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
   float* const seg_b = reinterpret_cast<float*>(dyn + a.off_segb);
   float* const seg_c = reinterpret_cast<float*>(dyn + a.off_segc);
   RowState& rs = sm.rs;
-  // The 2 * n_chunks segments this warp writes, in ascending token id: number i is piece i % 2 of
-  // chunk i / 2.  In the list passes group `grp` of 8 lanes takes numbers grp and grp + 4 (then
-  // + 8, ...), two segments side by side for instruction-level parallelism.
-  const int nsw = kPPW * a.n_chunks;
-  auto seg_of = [&](int i) { return (i >> 1) * kChunkPieces + (i & 1) * kSWarps + warp; };
 
   // this CTA's parents: [p_begin, p_end)
   const int p_begin = (int)(((long long)a.n_parents * blockIdx.x) / gridDim.x);
@@ -609,7 +606,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       uint4 rc[kPPW], ru[kPPW];
 #pragma unroll
       for (int i = 0; i < kPPW; ++i) {
-        const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
+        const int e = (kPPW * warp + i) * PIECE + lane * EPL;
         if (c * a.chunk + e < P.V) raw_load<BF16, ROW_U>(slot, a.chunk, e, rc[i], ru[i]);
       }
       release_slot();   // the data are in registers
@@ -617,7 +614,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       float z[kPPW][EPL];
 #pragma unroll
       for (int i = 0; i < kPPW; ++i) {
-        const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
+        const int e = (kPPW * warp + i) * PIECE + lane * EPL;
         mask[i] = 0;
         if (c * a.chunk + e < P.V) {
           raw_mix<BF16, ROW_U>(rc[i], ru[i], P.cfg_scale, P.invT, z[i]);
@@ -626,9 +623,9 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
             if (z[i][j] >= pivot) mask[i] |= 1u << j;
         }
       }
-      // one warp scan for both pieces' counts (16 bits each); lane 31 then claims one run of
-      // the row's array for the two segments, each rounded up to an even length so that the
-      // list passes can load entries in aligned pairs
+      // one warp scan for both pieces' counts (16 bits each); lane 31 then claims one run of the
+      // row's array for the segment (the two pieces back to back), rounded up to an even length
+      // so that runs start on even entries and the list passes can load aligned pairs
       static_assert(kPPW == 2, "the packed scan below handles two pieces");
       const unsigned cnt0 = __popc(mask[0]), cnt1 = __popc(mask[1]);
       unsigned inc = cnt0 | (cnt1 << 16);
@@ -638,15 +635,14 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         if (lane >= o) inc += t;
       }
       const unsigned tot = __shfl_sync(kFull, inc, 31);
-      const int t0 = (int)(tot & 0xffffu), t1 = (int)(tot >> 16);
-      const int t0e = (t0 + 1) & ~1, t1e = (t1 + 1) & ~1;
+      const int t0 = (int)(tot & 0xffffu), t01 = t0 + (int)(tot >> 16);
       int base = 0;
       if (lane == 31) {
-        base = (int)atomicAdd(&rs.alloc, (unsigned)(t0e + t1e));
-        const bool fits = base + t0e + t1e <= a.cap;
-        const int seg = c * kChunkPieces + warp;
-        run[seg] = make_ushort2((unsigned short)(fits ? base : 0), (unsigned short)(fits ? t0 : 0));
-        run[seg + kSWarps] = make_ushort2((unsigned short)(fits ? base + t0e : 0), (unsigned short)(fits ? t1 : 0));
+        const int len = (t01 + 1) & ~1;
+        base = (int)atomicAdd(&rs.alloc, (unsigned)len);
+        // (the draft row's look-up table holds offsets within a segment in 8 bits)
+        const bool fits = base + len <= a.cap && (!IS_Q || t01 <= 255);
+        run[c * kSWarps + warp] = make_ushort2((unsigned short)(fits ? base : 0), (unsigned short)(fits ? t01 : 0));
         if (!fits) {
           rs.overflow = 1;
           base = -1;
@@ -655,19 +651,19 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       base = __shfl_sync(kFull, base, 31);
 #pragma unroll
       for (int i = 0; i < kPPW; ++i) {
-        const int e = (i * kSWarps + warp) * PIECE + lane * EPL;
+        const int e = (kPPW * warp + i) * PIECE + lane * EPL;
         const int id0 = c * a.chunk + e;
-        const int off = i == 0 ? (int)(inc & 0xffffu) - (int)cnt0 : (int)(inc >> 16) - (int)cnt1;
-        const int b0 = i == 0 ? base : base + t0e;
+        // position of this lane's first candidate within the segment's run
+        const int off = i == 0 ? (int)(inc & 0xffffu) - (int)cnt0 : t0 + (int)(inc >> 16) - (int)cnt1;
         if (IS_Q && id0 < P.V) qcell[id0 / EPL] = (uint16_t)(mask[i] | ((unsigned)min(off, 255) << 8));
         if (base >= 0) {
           if (IS_Q) {
-            float* dst = qval + b0 + off;
+            float* dst = qval + base + off;
 #pragma unroll
             for (int j = 0; j < EPL; ++j)
               if ((mask[i] >> j) & 1u) *dst++ = z[i][j];
           } else {
-            uint2* dst = cand + b0 + off;
+            uint2* dst = cand + base + off;
 #pragma unroll
             for (int j = 0; j < EPL; ++j)
               if ((mask[i] >> j) & 1u) *dst++ = make_uint2(__float_as_uint(z[i][j]), (unsigned)(id0 + j));
@@ -675,8 +671,8 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         }
       }
     }
-    // ---- pass A over the lists this warp wrote: group `grp` of 8 lanes takes the warp's two
-    //      pieces of chunk grp, grp + 4, ...; a lane loads two neighbouring entries at a time
+    // ---- pass A over the lists this warp wrote; a lane takes two pairs of neighbouring entries
+    //      per trip, and the group's lanes cover 4 * seg_lanes entries of the segment
     __syncwarp();
     float mx = -INFINITY;
     unsigned mine = 0;
@@ -685,36 +681,25 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
       if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
     };
-    for (int iA = grp; iA < nsw; iA += 2 * kSegGroups) {
-      const int iB = iA + kSegGroups;
-      const ushort2 rA = run[seg_of(iA)], rB = iB < nsw ? run[seg_of(iB)] : make_ushort2(0, 0);
-      const int cnA = rA.y, cnB = rB.y;
-      if (sub == 0) mine += (unsigned)(cnA + cnB);
-      for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
-        if (sl < cnA) {
-          float z0, z1;
-          if (IS_Q) {
-            const float2 v = *reinterpret_cast<const float2*>(qval + rA.x + sl);
-            z0 = v.x, z1 = v.y;
-          } else {
-            const uint4 v = *reinterpret_cast<const uint4*>(cand + rA.x + sl);
-            z0 = __uint_as_float(v.x), z1 = __uint_as_float(v.z);
-          }
-          tally(z0);
-          if (sl + 1 < cnA) tally(z1);
-        }
-        if (sl < cnB) {
-          float z0, z1;
-          if (IS_Q) {
-            const float2 v = *reinterpret_cast<const float2*>(qval + rB.x + sl);
-            z0 = v.x, z1 = v.y;
-          } else {
-            const uint4 v = *reinterpret_cast<const uint4*>(cand + rB.x + sl);
-            z0 = __uint_as_float(v.x), z1 = __uint_as_float(v.z);
-          }
-          tally(z0);
-          if (sl + 1 < cnB) tally(z1);
-        }
+    auto tally_pair = [&](int first, int sl, int cn) {
+      float z0, z1;
+      if (IS_Q) {
+        const float2 v = *reinterpret_cast<const float2*>(qval + first + sl);
+        z0 = v.x, z1 = v.y;
+      } else {
+        const uint4 v = *reinterpret_cast<const uint4*>(cand + first + sl);
+        z0 = __uint_as_float(v.x), z1 = __uint_as_float(v.z);
+      }
+      tally(z0);
+      if (sl + 1 < cn) tally(z1);
+    };
+    for (int c = grp; c < a.n_chunks; c += groups) {
+      const ushort2 r = run[c * kSWarps + warp];
+      const int cn = r.y;
+      if (sub == 0) mine += (unsigned)cn;
+      for (int sl = 2 * sub; sl < cn; sl += 4 * seg_lanes) {
+        tally_pair(r.x, sl, cn);
+        if (sl + 2 * seg_lanes < cn) tally_pair(r.x, sl + 2 * seg_lanes, cn);
       }
     }
     __syncwarp();
@@ -826,31 +811,23 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         *reinterpret_cast<uint4*>(cand + at) = v;
       }
     };
-    for (int i0 = 0; i0 < nsw; i0 += 2 * kSegGroups) {
-      const int iA = i0 + grp, iB = iA + kSegGroups;
-      const bool hasA = iA < nsw, hasB = iB < nsw;
-      const int segA = seg_of(iA), segB = seg_of(iB);
-      float accA = 0.f, accB = 0.f;
-      if (hasA) {
-        const ushort2 rA = run[segA], rB = hasB ? run[segB] : make_ushort2(0, 0);
-        const int cnA = rA.y, cnB = rB.y;
-        for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
-          if (sl < cnA) pair(segA, rA, sl, accA);
-          if (sl < cnB) pair(segB, rB, sl, accB);
+    for (int c0 = 0; c0 < a.n_chunks; c0 += groups) {
+      const int c = c0 + grp;
+      const bool has = c < a.n_chunks;
+      const int seg = c * kSWarps + warp;
+      float acc = 0.f;
+      if (has) {
+        const ushort2 r = run[seg];
+        for (int sl = 2 * sub; sl < (int)r.y; sl += 4 * seg_lanes) {
+          pair(seg, r, sl, acc);
+          if (sl + 2 * seg_lanes < (int)r.y) pair(seg, r, sl + 2 * seg_lanes, acc);
         }
       }
       __syncwarp();
-      accA = seg_lanes_sum(accA);
-      accB = seg_lanes_sum(accB);
-      if (sub == 0) {
-        if (hasA) {
-          seg_a[segA] = accA;
-          if (!IS_Q) seg_c[segA] = accA;
-        }
-        if (hasB) {
-          seg_a[segB] = accB;
-          if (!IS_Q) seg_c[segB] = accB;
-        }
+      acc = seg_lanes_sum(acc, seg_lanes);
+      if (sub == 0 && has) {
+        seg_a[seg] = acc;
+        if (!IS_Q) seg_c[seg] = acc;
       }
     }
   };
@@ -1099,7 +1076,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
           const unsigned cell = qcell[id / EPL];
           const int j = id % EPL;
           float qe = 0.f;
-          if ((cell >> j) & 1u) qe = qval[(int)qseg[id / PIECE].x + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
+          if ((cell >> j) & 1u) qe = qval[(int)qseg[id / SEG].x + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
           return fmaxf(__fsub_rn(pe, __fmul_rn(qe, invZq)), 0.f);
         };
         auto w_resid = [&](int i) {
@@ -1114,26 +1091,21 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         };
         auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
         if (draws & kDrawResidual) {   // block-uniform
-          for (int i0 = 0; i0 < nsw; i0 += 2 * kSegGroups) {
-            const int iA = i0 + grp, iB = iA + kSegGroups;
-            const bool hasA = iA < nsw, hasB = iB < nsw;
-            const int segA = seg_of(iA), segB = seg_of(iB);
-            float accA = 0.f, accB = 0.f;
-            if (hasA) {
-              const ushort2 rA = tseg[segA], rB = hasB ? tseg[segB] : make_ushort2(0, 0);
-              const int cnA = rA.y, cnB = rB.y;
-              for (int sl = 2 * sub; sl < max(cnA, cnB); sl += 2 * kSegLanes) {
-                if (sl < cnA) accA += w_pair(rA, sl);
-                if (sl < cnB) accB += w_pair(rB, sl);
+          for (int c0 = 0; c0 < a.n_chunks; c0 += groups) {
+            const int c = c0 + grp;
+            const bool has = c < a.n_chunks;
+            const int seg = c * kSWarps + warp;
+            float acc = 0.f;
+            if (has) {
+              const ushort2 r = tseg[seg];
+              for (int sl = 2 * sub; sl < (int)r.y; sl += 4 * seg_lanes) {
+                acc += w_pair(r, sl);
+                if (sl + 2 * seg_lanes < (int)r.y) acc += w_pair(r, sl + 2 * seg_lanes);
               }
             }
             __syncwarp();
-            accA = seg_lanes_sum(accA);
-            accB = seg_lanes_sum(accB);
-            if (sub == 0) {
-              if (hasA) seg_b[segA] = accA;
-              if (hasB) seg_b[segB] = accB;
-            }
+            acc = seg_lanes_sum(acc, seg_lanes);
+            if (sub == 0 && has) seg_b[seg] = acc;
           }
         }
         __syncthreads();

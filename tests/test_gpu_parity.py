@@ -283,7 +283,9 @@ def test_identity_fast_path(ctx):
     batch = pu.build_batch(cfg)
     g = pu.gpu_round(ctx, cfg, batch)
     assert ctx.poll_device_status() == 0
-    assert g["n_reject"].sum() == 0 and np.all(g["accept_prob"] == 1.0)
+    # the two partition sums are added up in an order that depends on each row's own pivot, so
+    # p / q may miss 1 by a rounding error of the fp32 segment sums
+    assert g["n_reject"].sum() == 0 and np.all(np.abs(g["accept_prob"] - 1.0) <= 1e-6)
     assert np.array_equal(g["out_tok"], batch["tok_lo"].cpu().numpy().repeat(2, 1).repeat(2, 2))
 
 
