@@ -184,6 +184,7 @@ inline size_t stream_layout(StreamArgs& a, int esz) {
 struct Predictor {
   int have;
   float theta, rho;
+  float pivot, inv_w;   // what the next row of this kind starts from (valid while have != 0)
   // rows without a prediction take the pivot from the mean and spread of their first chunk,
   // assuming a normal shape; when that start fails, `shift` (in units of the spread) moves the
   // next start down (too few candidates) or up (too many): the step doubles while the
@@ -460,6 +461,8 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       sm.pred[s].have = 0;
       sm.pred[s].theta = 0.f;
       sm.pred[s].rho = 1.f;
+      sm.pred[s].pivot = 0.f;
+      sm.pred[s].inv_w = 0.f;
       sm.pred[s].shift = 0.f;
       sm.pred[s].step = 0.f;
       sm.pred[s].dir = 0;
@@ -540,9 +543,8 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     constexpr bool ROW_U = decltype(has_u_tag)::value;
     const Predictor pr = sm.pred[kind];
     if (pr.have) {   // block-uniform
-      const float d = (float)a.margin / pr.rho;
-      pivot = pr.theta - d;
-      inv_w = (float)kHistBins / (3.0f * d);
+      pivot = pr.pivot;
+      inv_w = pr.inv_w;
       return;
     }
     mbar_wait(&sm.full[rslot], rphase, a.dev_status);
@@ -914,6 +916,11 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         pr.theta = pr.have ? pr.theta + 0.25f * (theta - pr.theta) : theta;
         pr.rho = rho;
         pr.have = 1;
+        // the next row's pivot: `margin` entries' worth below the predicted threshold; its
+        // histogram spans three times that distance
+        const float d = (float)a.margin / rho;
+        pr.pivot = pr.theta - d;
+        pr.inv_w = (float)kHistBins / (3.0f * d);
       }
     }
     sm.pred[kind] = pr;
