@@ -1077,23 +1077,25 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
           defer(g);
         }
         // weight of candidate i in the residual of Eq. 2 (lambda = 1)
-        auto w_entry = [&](unsigned ebits, unsigned idbits) {
+        // (every token id of a target segment lies in the draft row's segment of the same
+        // number, whose run starts at entry `qfirst` of the draft list)
+        auto w_entry = [&](unsigned ebits, unsigned idbits, int qfirst) {
           const float pe = __fmul_rn(__uint_as_float(ebits), invZp);
           const int id = (int)idbits;
           const unsigned cell = qcell[id / EPL];
           const int j = id % EPL;
           float qe = 0.f;
-          if ((cell >> j) & 1u) qe = qval[(int)qseg[id / SEG].x + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
+          if ((cell >> j) & 1u) qe = qval[qfirst + (int)(cell >> 8) + __popc(cell & ((1u << j) - 1u))];
           return fmaxf(__fsub_rn(pe, __fmul_rn(qe, invZq)), 0.f);
         };
         auto w_resid = [&](int i) {
           const uint2 en = cand[i];
-          return w_entry(en.x, en.y);
+          return w_entry(en.x, en.y, (int)qseg[(int)en.y / SEG].x);
         };
-        auto w_pair = [&](ushort2 r, int sl) {
+        auto w_pair = [&](ushort2 r, int sl, int qfirst) {
           const uint4 v = *reinterpret_cast<const uint4*>(cand + r.x + sl);
-          float w = w_entry(v.x, v.y);
-          if (sl + 1 < r.y) w += w_entry(v.z, v.w);
+          float w = w_entry(v.x, v.y, qfirst);
+          if (sl + 1 < r.y) w += w_entry(v.z, v.w, qfirst);
           return w;
         };
         auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
@@ -1105,9 +1107,10 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
             float acc = 0.f;
             if (has) {
               const ushort2 r = tseg[seg];
+              const int qfirst = qseg[seg].x;
               for (int sl = 2 * sub; sl < (int)r.y; sl += 4 * seg_lanes) {
-                acc += w_pair(r, sl);
-                if (sl + 2 * seg_lanes < (int)r.y) acc += w_pair(r, sl + 2 * seg_lanes);
+                acc += w_pair(r, sl, qfirst);
+                if (sl + 2 * seg_lanes < (int)r.y) acc += w_pair(r, sl + 2 * seg_lanes, qfirst);
               }
             }
             __syncwarp();
