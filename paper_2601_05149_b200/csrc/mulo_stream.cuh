@@ -958,6 +958,15 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     pp.z_tok = load1(tr, sm.tok);
   };
 
+  // One thread, a phase ahead of prepare_row: asks L2 for the lines that hold the logit of x~ at
+  // the next target position, so that the load there does not wait on HBM.
+  auto prefetch_row = [&](int child) {
+    const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
+    const size_t off = (((size_t)sm.b * P.H * P.W + t) * (size_t)P.V + (size_t)sm.tok) * esz;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.cond + off));
+    if (HAS_U) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.uncond + off));
+  };
+
   for (int parent = p_begin; parent < p_end; ++parent) {
     // ------------------------------------------------------------ draft row
     {
@@ -985,6 +994,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       choose_pivot(0, std::false_type{}, pivot, inv_w);
       stream_row(std::true_type{}, std::false_type{}, pivot, inv_w);
       __syncthreads();
+      if (tid == 64) prefetch_row(0);
       Sel s;
       bool ok = locate_bin(s);
       float theta = 0.f;
@@ -1032,6 +1042,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         choose_pivot(1, std::integral_constant<bool, HAS_U>{}, pivot, inv_w);
         stream_row(std::false_type{}, std::integral_constant<bool, HAS_U>{}, pivot, inv_w);
         __syncthreads();
+        if (tid == 64 && child + 1 < rr) prefetch_row(child + 1);
         Sel s;
         bool ok = locate_bin(s);
         if (ok) {
