@@ -886,7 +886,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     return true;
   };
 
-  // Thread 0: the predictor of a kind of row after a row (ok: theta found exactly).
+  // One thread: the predictor of a kind of row after a row (ok: theta found exactly).
   auto learn = [&](int kind, bool ok, int reason, float theta, float pivot, int n, int n_ge) {
     Predictor pr = sm.pred[kind];
     if (!ok) {
@@ -944,15 +944,19 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     atomicAdd(a.dev_status + kCntRows, 1u);
   };
 
-  // One thread: the uniforms of a target position and the logit of x~ there.
-  auto prepare_row = [&](RowPrep& pp, int child) {
+  // Two threads of different warps: the uniforms of a target position (`part` 0) and the
+  // logit of x~ there (`part` 1).
+  auto prepare_row = [&](RowPrep& pp, int child, int part) {
     const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
     const size_t g = (size_t)sm.b * P.H * P.W + t;
-    const uint4 r = philox4x32_10(make_uint4((uint32_t)t, (uint32_t)sm.b + P.image_offset, P.round, 0u),
-                                  make_uint2(P.seed_lo, P.seed_hi));
-    pp.rnd[0] = r.x;
-    pp.rnd[1] = r.y;
-    pp.rnd[2] = r.z;
+    if (part == 0) {
+      const uint4 r = philox4x32_10(make_uint4((uint32_t)t, (uint32_t)sm.b + P.image_offset, P.round, 0u),
+                                    make_uint2(P.seed_lo, P.seed_hi));
+      pp.rnd[0] = r.x;
+      pp.rnd[1] = r.y;
+      pp.rnd[2] = r.z;
+      return;
+    }
     RowSrc tr = {a.cond + g * (size_t)P.V * esz, HAS_U ? a.uncond + g * (size_t)P.V * esz : nullptr, P.cfg_scale,
                  P.invT, P.V, BF16};
     pp.z_tok = load1(tr, sm.tok);
@@ -1027,7 +1031,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       }
       __syncthreads();   // everybody is done with the selection scratch
       reset_state();
-      if (tid == 64 && ok) prepare_row(sm.prep[rowi & 1], 0);   // first child's uniforms and logit of x~
+      if ((tid == 64 || tid == 96) && ok) prepare_row(sm.prep[rowi & 1], 0, tid == 96);   // first child's uniforms and logit of x~
       __syncthreads();
     }
 
@@ -1054,7 +1058,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         int n_ge = 0;
         double Zp = 1.0;
         if (ok) ok = finish_selection(std::false_type{}, s, theta, n_ge, Zp);
-        if (tid == 0) learn(1, ok, s.reason, theta, pivot, s.n, n_ge);
+        const bool ok_sel = ok;   // the predictor learns from it while the draws run
         const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
         const size_t g = (size_t)sm.b * P.H * P.W + t;
         int draws = 0;
@@ -1150,7 +1154,8 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
             if (lane == 0) a.cand_tgt[g] = t_tgt;
           }
         }
-        if (tid == 64 && child + 1 < rr) prepare_row(sm.prep[(rowi + 1) & 1], child + 1);
+        if ((tid == 64 || tid == 96) && child + 1 < rr) prepare_row(sm.prep[(rowi + 1) & 1], child + 1, tid == 96);
+        if (tid == 128) learn(1, ok_sel, s.reason, theta, pivot, s.n, n_ge);
         ++rowi;
         __syncthreads();
       }
