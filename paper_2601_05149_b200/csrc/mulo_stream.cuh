@@ -628,8 +628,8 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       // one warp scan for both pieces' counts (16 bits each); lane 31 then claims one run of the
       // row's array for the segment (the two pieces back to back), rounded up to an even length
       // so that runs start on even entries and the list passes can load aligned pairs
-      static_assert(kPPW == 2, "the packed scan below handles two pieces");
-      const unsigned cnt0 = __popc(mask[0]), cnt1 = __popc(mask[1]);
+      static_assert(kPPW <= 2, "the packed scan below handles at most two pieces");
+      const unsigned cnt0 = __popc(mask[0]), cnt1 = kPPW > 1 ? __popc(mask[kPPW - 1]) : 0u;
       unsigned inc = cnt0 | (cnt1 << 16);
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
