@@ -72,6 +72,7 @@ def lib() -> C.CDLL:
             _lib.orc_accept_threshold.argtypes = [C.c_double, C.c_double]
             _lib.orc_inverse_cdf.restype = C.c_int
             _lib.orc_expand.restype = C.c_int
+            _lib.orc_islands.restype = C.c_int
     return _lib
 
 
@@ -179,6 +180,18 @@ def expand(reject, radius, clip_before_first=1):
     out = np.empty_like(reject)
     t0 = lib().orc_expand(_ptr(reject), H, W, int(radius), int(clip_before_first), _ptr(out))
     return out, int(t0)
+
+
+def islands(in_rx):
+    """Eq. 8: labels [H, W] (0 outside R_X, islands 1..M numbered by their first raster
+    position), and per island its first / last grid row and its number of positions."""
+    in_rx = np.ascontiguousarray(in_rx, np.uint8)
+    H, W = in_rx.shape
+    labels = np.zeros((H, W), np.int32)
+    rows = np.zeros((max(H * W, 1), 2), np.int32)
+    size = np.zeros(max(H * W, 1), np.int32)
+    M = int(lib().orc_islands(_ptr(in_rx), H, W, _ptr(labels), _ptr(rows), _ptr(size)))
+    return labels, M, rows[:M].copy(), size[:M].copy()
 
 
 def position_distributions(params, cond_row, uncond_row, draft_row, tok, nn=None):

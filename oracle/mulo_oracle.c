@@ -19,6 +19,7 @@
  *   Sec. 3.3 Eq. 6   N(t,l) = {u : |i_u-i_t|<=l, |j_u-j_t|<=l, u >= t_0}
  *   Sec. 3.3 Eq. 7   R_X = union of N(t,l) over rejected t
  *   Algorithm 1      Step 4 (accept), Step 5 (expand), Step 6 (resample from M_p)
+ *   Sec. 3.4 Eq. 8   rejection islands {I_m} = CC_8(R_X): 8-connected components
  *   Supp. "Sampling" temperature, top-k, classifier-free guidance of the sampler
  *
  * Readings taken where the paper is silent (each is listed in the design notes):
@@ -47,8 +48,10 @@
  * torch in fp64; target == draft accepts everything; E[accept] = sum min(p,q);
  * residual mass = TVD; exact output pmf by enumeration of all 2^24 uniforms;
  * chi-square of the whole round; dilation against scipy and brute force;
- * inverse CDF against numpy.searchsorted.  The paper prints no worked numeric
- * example for this path, so no pin is a printed value.
+ * inverse CDF against numpy.searchsorted; islands against scipy.ndimage.label,
+ * against reachability by boolean matrix closure on every mask of a small grid,
+ * and on hand-drawn shapes.  The paper prints no worked numeric example for this
+ * path, so no pin is a printed value.
  */
 #include <math.h>
 #include <stdint.h>
@@ -311,6 +314,53 @@ int orc_expand(const uint8_t* reject, int H, int W, int radius, int clip_before_
     }
   }
   return t0;
+}
+
+/* Eq. 8: the rejection islands are the classes of R_X under "joined by a chain
+ * of positions of R_X in which consecutive positions differ by at most 1 in
+ * both coordinates".  Written out as that definition: walk the grid in raster
+ * order; a position of R_X that has no island yet opens island m = M + 1 and
+ * everything reachable from it through 8-neighbours gets m.  Islands are thereby
+ * numbered by the raster index of their first position (a convention of this
+ * code; the paper leaves the numbering open).
+ *   in_rx   [H*W] bytes (0/1);  labels [H*W] out, 0 outside R_X;
+ *   rows    [H*W][2] out: first and last grid row of islands 1..M (entry m-1);
+ *   size    [H*W]    out: number of positions.   Returns M. */
+int orc_islands(const uint8_t* in_rx, int H, int W, int32_t* labels, int32_t* rows, int32_t* size) {
+  const int N = H * W;
+  if (H <= 0 || W <= 0) return 0;
+  int32_t* stack = (int32_t*)malloc(sizeof(int32_t) * (size_t)N);
+  int M = 0;
+  for (int t = 0; t < N; ++t) labels[t] = 0;
+  for (int t = 0; t < N; ++t) {
+    if (!in_rx[t] || labels[t]) continue;
+    ++M;
+    int top = 0;
+    stack[top++] = t;
+    labels[t] = M;
+    rows[2 * (M - 1)] = t / W;
+    rows[2 * (M - 1) + 1] = t / W;
+    size[M - 1] = 0;
+    while (top > 0) {
+      const int v = stack[--top];
+      const int iv = v / W, jv = v % W;
+      size[M - 1] += 1;
+      if (iv < rows[2 * (M - 1)]) rows[2 * (M - 1)] = iv;
+      if (iv > rows[2 * (M - 1) + 1]) rows[2 * (M - 1) + 1] = iv;
+      for (int di = -1; di <= 1; ++di)
+        for (int dj = -1; dj <= 1; ++dj) {
+          const int iu = iv + di, ju = jv + dj;
+          if ((di == 0 && dj == 0) || iu < 0 || iu >= H || ju < 0 || ju >= W) continue;
+          const int u = iu * W + ju;
+          if (in_rx[u] && !labels[u]) {
+            labels[u] = M;
+            stack[top++] = u;
+          }
+        }
+    }
+  }
+  free(stack);
+  return M;
 }
 
 /* ---------------------------------------------------------------- stages */
