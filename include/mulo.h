@@ -12,6 +12,7 @@
  *   -> rejection mask R_T, first rejection t_0       (Sec. 3.3)
  *   -> local expansion R_X                           (Sec. 3.3, Eq. 6-7)
  *   -> parallel inverse-CDF redraw of R_X            (Eq. 2; Algorithm 1 Step 6)
+ * and, for the scheduler of the redraw, the rejection islands of R_X (Sec. 3.4, Eq. 8).
  *
  * Conventions for every call
  *   - All tensor arguments are DEVICE pointers to caller-owned, contiguous,
@@ -190,6 +191,25 @@ mulo_status mulo_verify(mulo_ctx* ctx, const mulo_params* p, const void* tgt_con
 mulo_status mulo_local_reject_expand(mulo_ctx* ctx, const mulo_params* p,
                                      const uint32_t* reject_bits, const int32_t* first_reject,
                                      uint32_t* expand_bits, int32_t* n_expand, void* stream);
+
+/* Rejection islands (Sec. 3.4, Eq. 8): {I_m} = CC_8(R_X), the 8-connected components of R_X
+ * on the token grid (two positions are neighbours when both coordinates differ by at most
+ * one), which a scheduler redraws concurrently.  Uses B, H, W of `p`; H * W <= 16384, else
+ * MULO_ERR_UNSUPPORTED.  Needs no workspace.
+ *   expand_bits [B, H, ceil(W/32)]   in   R_X
+ *   labels      [B, H, W]            out  0 outside R_X, else the island's number m in 1..M.
+ *                                         Islands are numbered by the raster index of their
+ *                                         first position (the paper leaves the order open).
+ *   n_islands   [B]                  out  M
+ *   max_islands                           rows of the two tables below per image (>= 0)
+ *   island_rows [B, max_islands, 2]  out, may be NULL: first and last grid row of island m at
+ *                                         entry m - 1; entries from M on are (-1, -1)
+ *   island_size [B, max_islands]     out, may be NULL: number of positions; 0 from M on
+ * With M > max_islands the labels and n_islands are still complete; the tables hold the
+ * first max_islands islands. */
+mulo_status mulo_islands(mulo_ctx* ctx, const mulo_params* p, const uint32_t* expand_bits,
+                         int32_t* labels, int32_t* n_islands, int32_t max_islands,
+                         int32_t* island_rows, int32_t* island_size, void* stream);
 
 /* Step 6 on given logits: every position of R_X is redrawn in parallel by inverse CDF over
  * w(x) = max(0, p'(x) - lambda q(x)) in ascending token id, lambda = 1 (Eq. 2) or 0

@@ -24,7 +24,7 @@ EXPORTS = (
     "mulo_create", "mulo_destroy", "mulo_status_string", "mulo_workspace_bytes",
     "mulo_set_workspace", "mulo_poll_device_status", "mulo_poll_fallback_counts", "mulo_kernel_launches",
     "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only",
-    "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_resample",
+    "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_islands", "mulo_resample",
     "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host", "mulo_round_static",
 )
 
@@ -218,6 +218,18 @@ class Context:
         _check(lib().mulo_local_reject_expand(self._ctx, C.byref(p), _dev(reject_bits),
                                               _dev(first_reject), _dev(expand_bits), _dev(n_expand),
                                               _stream(stream)), "mulo_local_reject_expand")
+
+    def mulo_islands(self, p, expand_bits, labels, n_islands, island_rows=None, island_size=None,
+                     max_islands=None, stream=None):
+        if max_islands is None:
+            max_islands = 0
+            if island_rows is not None:
+                max_islands = island_rows.shape[1]
+            elif island_size is not None:
+                max_islands = island_size.shape[1]
+        _check(lib().mulo_islands(self._ctx, C.byref(p), _dev(expand_bits), _dev(labels), _dev(n_islands),
+                                  C.c_int32(int(max_islands)), _dev(island_rows), _dev(island_size),
+                                  _stream(stream)), "mulo_islands")
 
     def mulo_resample(self, p, tgt_cond, tgt_uncond, draft_logits_lo, draft_stats_lo, draft_tok_hi, nn,
                       reject_bits, expand_bits, out_tok, stream=None):

@@ -10,6 +10,7 @@
 
 #include "../../include/mulo.h"
 #include "mulo_dense.cuh"
+#include "mulo_islands.cuh"
 #include "mulo_stream.cuh"
 
 using namespace mulo;
@@ -780,6 +781,31 @@ mulo_status mulo_local_reject_expand(mulo_ctx* ctx, const mulo_params* p, const 
   m.reject_in = reject_bits; m.first_in = first_reject;
   m.expand_bits = expand_bits; m.n_expand = n_expand;
   k_mask<1><<<p->B, kMaskThreads, mask_smem(p), (cudaStream_t)stream>>>(m);
+  return launched(ctx, 1);
+}
+
+mulo_status mulo_islands(mulo_ctx* ctx, const mulo_params* p, const uint32_t* expand_bits, int32_t* labels,
+                         int32_t* n_islands, int32_t max_islands, int32_t* island_rows,
+                         int32_t* island_size, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!expand_bits || !labels || !n_islands || max_islands < 0) return MULO_ERR_INVALID_ARG;
+  if ((size_t)p->H * p->W > (size_t)kIslandMaxCells) return MULO_ERR_UNSUPPORTED;
+  if (p->B == 0) return MULO_OK;
+  IslandArgs a;
+  a.H = p->H; a.W = p->W; a.max_islands = max_islands;
+  a.bits = expand_bits; a.labels = labels; a.n_islands = n_islands;
+  a.rows = max_islands > 0 ? island_rows : nullptr;
+  a.size = max_islands > 0 ? island_size : nullptr;
+  const size_t smem = ((size_t)2 * p->H * p->W + (size_t)p->H * ((p->W + 31) / 32)) * sizeof(int);
+  if (smem + 1024 > (size_t)ctx->smem_optin) return MULO_ERR_UNSUPPORTED;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(k_islands, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return MULO_ERR_CUDA;
+  }
+  k_islands<<<p->B, kIslandThreads, smem, (cudaStream_t)stream>>>(a);
   return launched(ctx, 1);
 }
 
