@@ -399,6 +399,75 @@ def run_sweep(args):
     ctx.close()
 
 
+def run_islands(args, cfg):
+    """Rejection islands (Eq. 8) of the masks one round of the workload leaves: one JSON line per batch size
+    (the workload's own batch, then the same masks repeated to 1024 images), with the CPU oracle timed on the
+    same masks.  Single GPU."""
+    from paper_2601_05149_b200 import binding
+    import numpy as np
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the islands kernel has no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    ctx = binding.Context(0)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else 6650.0
+    batch = synth.build_batch(cfg, dev)
+    p = binding.params_from_config(cfg)
+    ctx.ensure_workspace(p)
+    out = binding.alloc_round_outputs(p, dev, probs=False)
+    ctx.mulo_round(p, batch["cond"], batch["uncond"], batch["draft_lo"], batch["tok_lo"], batch["nn"],
+                   out["out_tok"], out["reject_bits"], out["expand_bits"], None, None, None,
+                   out["n_reject"], out["n_expand"], out["first_reject"])
+    torch.cuda.synchronize()
+    del batch
+    W, K = max(3, args.warmup), max(1, args.steps)
+    cap = 256
+    for B in (cfg.B, max(cfg.B, 1024)):
+        reps = (B + cfg.B - 1) // cfg.B
+        bits = out["expand_bits"].repeat(reps, 1, 1)[:B].contiguous()
+        pb = binding.params_from_config(dataclasses.replace(cfg, B=B))
+        labels = torch.empty((B, cfg.H, cfg.W), dtype=torch.int32, device=dev)
+        n = torch.empty((B,), dtype=torch.int32, device=dev)
+        rows = torch.empty((B, cap, 2), dtype=torch.int32, device=dev)
+        size = torch.empty((B, cap), dtype=torch.int32, device=dev)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+        launches0 = ctx.kernel_launches()
+        e = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for s_ in range(W + K):
+            flush.zero_()
+            if s_ >= W:
+                e[s_ - W][0].record()
+            ctx.mulo_islands(pb, bits, labels, n, rows, size)
+            if s_ >= W:
+                e[s_ - W][1].record()
+        torch.cuda.synchronize()
+        ms = statistics.mean(a.elapsed_time(b) for a, b in e)
+        positions = B * cfg.H * cfg.W
+        alg = bits.numel() * 4 + labels.numel() * 4 + n.numel() * 4 + rows.numel() * 4 + size.numel() * 4
+        cpu = None
+        if B == cfg.B and not args.no_cpu_baseline:
+            import oracle
+            masks = binding.unpack_bits(bits, cfg.W).numpy().astype(np.uint8)
+            t0 = time.time()
+            total = sum(oracle.islands(masks[b])[1] for b in range(B))
+            dt = time.time() - t0
+            assert total == int(n.sum().item())
+            cpu = {"value": positions / dt, "unit": "positions/s", "cores": 1, "kind": "oracle",
+                   "sample": f"all {B} masks of the batch", "seconds": dt}
+        print(json.dumps({
+            "stage": "mulo_islands", "metric": "island_labelled_positions_per_sec",
+            "value": positions / (ms * 1e-3), "unit": "positions/s", "ms_per_step": ms, "steps": K, "warmup": W,
+            "dtype": "int32", "data": "synthetic",
+            "config": {"workload": workload_desc(cfg), "images": B, "islands_per_image": int(n.sum().item()) / B,
+                       "l2": "256 MB written between timed launches"},
+            "roofline": {"bound": "hbm", "kernel": "k_islands", "achieved": alg / (ms * 1e-3) / 1e9, "peak": peak,
+                         "unit": "GB/s", "frac": alg / (ms * 1e-3) / 1e9 / peak, "bytes_per_launch": alg,
+                         "traffic": None},
+            "cpu_baseline": cpu, "gpu_launches": ctx.kernel_launches() - launches0}), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,12 +479,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the bench line")
     ap.add_argument("--sweep-limit", type=int, default=0, help="only the first N sweep points")
+    ap.add_argument("--islands", action="store_true",
+                    help="time the rejection-island labelling of the workload's masks instead of the bench line")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.workload]
     if args.batch:
         cfg = dataclasses.replace(cfg, B=args.batch, name=f"{cfg.name}(B={args.batch})")
     if args.sweep:
         run_sweep(args)
+    elif args.islands:
+        run_islands(args, cfg)
     elif args.impl == "reference":
         run_reference(args, cfg)
     else:

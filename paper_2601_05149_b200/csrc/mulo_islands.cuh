@@ -3,11 +3,13 @@
 //
 // The grid of one image (at most kIslandMaxCells positions) lives in shared memory as a
 // forest: parent[t] is an earlier raster index of the same island, a root points at itself.
-// Every position of R_X is joined with its already-scanned neighbours (west; north, or
-// north-west and north-east when north is not in R_X: with north present those two are
-// joined to it by their own west/east links).  Joining hangs the later root under the earlier
-// one with atomicMin, so the root of an island is its first raster position; numbering the
-// roots in raster order (a block-wide count) numbers the islands by their first position.
+// Horizontal links cost nothing: every position starts out pointing at the first position of
+// its run of consecutive R_X bits in the row, found with bit operations on the mask words.
+// Only the first position of a run then works: it joins its run with every run of the row
+// above that reaches into columns [first - 1, last + 1].  Joining hangs the later root under
+// the earlier one with atomicMin, so the root of an island is its first raster position;
+// numbering the roots in raster order (a block-wide count) numbers the islands by their
+// first position.
 #pragma once
 #include <cstdint>
 
@@ -63,31 +65,91 @@ __global__ void __launch_bounds__(kIslandThreads) k_islands(IslandArgs a) {
   __shared__ int s_carry;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  for (int w = tid; w < nw; w += kIslandThreads) word[w] = a.bits[(size_t)b * nw + w];
+  for (int w = tid; w < nw; w += kIslandThreads) {
+    uint32_t v = a.bits[(size_t)b * nw + w];
+    if (w % Ww == Ww - 1 && (W & 31)) v &= (1u << (W & 31)) - 1u;   // bits past the row's end do not count
+    word[w] = v;
+  }
   if (tid == 0) s_carry = 0;
   __syncthreads();
+  // t = i * W + j without an integer division (t < 2^14: the float quotient is off by one at most)
+  const float inv_w = 1.0f / (float)W;
+  auto split = [&](int t, int& i, int& j) {
+    i = (int)((float)t * inv_w);
+    j = t - i * W;
+    if (j < 0) {
+      --i;
+      j += W;
+    } else if (j >= W) {
+      ++i;
+      j -= W;
+    }
+  };
   auto in_rx = [&](int i, int j) -> bool {
     return i >= 0 && j >= 0 && j < W && ((word[i * Ww + (j >> 5)] >> (j & 31)) & 1u);
   };
-  for (int t = tid; t < N; t += kIslandThreads) parent[t] = in_rx(t / W, t % W) ? t : -1;
+  // first column of the run of R_X bits that holds (i, j); (i, j) itself is in R_X
+  auto run_first = [&](int i, int j) -> int {
+    int w = j >> 5;
+    uint32_t gaps = ~word[i * Ww + w] & ((1u << (j & 31)) - 1u);   // zeros below j in its word
+    while (gaps == 0u && w > 0) {
+      --w;
+      gaps = ~word[i * Ww + w];
+    }
+    return gaps ? (w << 5) + 32 - __clz(gaps) : 0;
+  };
+  // last column of the run that starts at (i, j)
+  auto run_last = [&](int i, int j) -> int {
+    int w = j >> 5;
+    uint32_t gaps = ~word[i * Ww + w] & ~((2u << (j & 31)) - 1u);   // zeros above j in its word
+    while (gaps == 0u && w + 1 < Ww) {
+      ++w;
+      gaps = ~word[i * Ww + w];
+    }
+    return gaps ? (w << 5) + __ffs(gaps) - 2 : W - 1;
+  };
+  for (int t = tid; t < N; t += kIslandThreads) {
+    int i, j;
+    split(t, i, j);
+    parent[t] = in_rx(i, j) ? i * W + run_first(i, j) : -1;
+  }
   __syncthreads();
 
   for (int t = tid; t < N; t += kIslandThreads) {
-    const int i = t / W, j = t % W;
-    if (!in_rx(i, j)) continue;
-    if (in_rx(i, j - 1)) island_join(parent, t, t - 1);
-    if (in_rx(i - 1, j)) {
-      island_join(parent, t, t - W);
-    } else {
-      if (in_rx(i - 1, j - 1)) island_join(parent, t, t - W - 1);
-      if (in_rx(i - 1, j + 1)) island_join(parent, t, t - W + 1);
+    int i, j;
+    split(t, i, j);
+    if (i == 0 || !in_rx(i, j) || in_rx(i, j - 1)) continue;   // only the first position of a run works
+    const int last = run_last(i, j);
+    // runs of the row above inside columns [lo, hi]: one join per run, at its first bit there
+    const int lo = j > 0 ? j - 1 : 0, hi = last + 1 < W ? last + 1 : W - 1;
+    for (int w = lo >> 5; w <= hi >> 5; ++w) {
+      uint32_t up = word[(i - 1) * Ww + w];
+      uint32_t below = w > (lo >> 5) ? word[(i - 1) * Ww + w - 1] >> 31 : 0u;   // bit left of this word
+      if (w == lo >> 5) up &= ~((1u << (lo & 31)) - 1u);
+      if (w == hi >> 5 && (hi & 31) != 31) up &= (2u << (hi & 31)) - 1u;
+      uint32_t firsts = up & ~((up << 1) | below);   // first bit, inside the window, of each run
+      while (firsts) {
+        const int x = (w << 5) + __ffs(firsts) - 1;
+        firsts &= firsts - 1u;
+        island_join(parent, t, (i - 1) * W + x);
+      }
     }
   }
   __syncthreads();
-  // every position points straight at its root (a reader that meets a half-updated chain
-  // still walks to the same root)
-  for (int t = tid; t < N; t += kIslandThreads)
-    if (parent[t] >= 0) parent[t] = island_root(parent, t);
+  // first positions of runs point straight at their root (a reader that meets a half-updated
+  // chain still walks to the same root); then everybody else, one hop behind
+  for (int t = tid; t < N; t += kIslandThreads) {
+    int i, j;
+    split(t, i, j);
+    if (parent[t] >= 0 && !in_rx(i, j - 1)) parent[t] = island_root(parent, t);
+  }
+  __syncthreads();
+  for (int t = tid; t < N; t += kIslandThreads) {
+    int i, j;
+    split(t, i, j);
+    const int q = parent[t];
+    if (q >= 0 && in_rx(i, j - 1)) parent[t] = parent[q];
+  }
   __syncthreads();
 
   // number the roots in raster order
@@ -97,12 +159,17 @@ __global__ void __launch_bounds__(kIslandThreads) k_islands(IslandArgs a) {
     const unsigned roots = __ballot_sync(0xffffffffu, is_root);
     if (lane == 0) s_warp[warp] = __popc(roots);
     __syncthreads();
-    int before = s_carry, total = 0;
-    for (int w = 0; w < kIslandThreads / 32; ++w) {
-      const int c = s_warp[w];
-      if (w < warp) before += c;
-      total += c;
+    // every warp scans the 32 warp counts
+    static_assert(kIslandThreads == 1024, "one count per lane");
+    const int mine = s_warp[lane];
+    int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
     }
+    const int before = s_carry + __shfl_sync(0xffffffffu, inc - mine, warp);
+    const int total = __shfl_sync(0xffffffffu, inc, 31);
     if (is_root) number[t] = before + __popc(roots & ((1u << lane) - 1u)) + 1;
     __syncthreads();
     if (tid == 0) s_carry += total;
@@ -126,12 +193,14 @@ __global__ void __launch_bounds__(kIslandThreads) k_islands(IslandArgs a) {
     const int root = parent[t];
     const int m = root >= 0 ? number[root] : 0;
     a.labels[(size_t)b * N + t] = m;
-    if (m > 0 && m <= cap) {
+    int i, j;
+    split(t, i, j);
+    if (m > 0 && m <= cap && !in_rx(i, j - 1)) {   // one contribution per run of the row
       if (rows) {
-        atomicMin(&rows[2 * (m - 1)], t / W);
-        atomicMax(&rows[2 * (m - 1) + 1], t / W);
+        atomicMin(&rows[2 * (m - 1)], i);
+        atomicMax(&rows[2 * (m - 1) + 1], i);
       }
-      if (size) atomicAdd(&size[m - 1], 1);
+      if (size) atomicAdd(&size[m - 1], run_last(i, j) - j + 1);
     }
   }
 }
