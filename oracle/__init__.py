@@ -207,11 +207,21 @@ def position_distributions(params, cond_row, uncond_row, draft_row, tok, nn=None
     return q, p, pp, mass.value
 
 
-def sample_draft_tokens(params, draft_lo):
+def sample_draft_tokens(params, draft_lo, with_edge=False):
     h, w = params.H // params.r, params.W // params.r
     tok = np.empty((h, w), np.int32)
-    lib().orc_sample_draft_tokens(C.byref(params), _ptr(np.ascontiguousarray(draft_lo)), _ptr(tok))
-    return tok
+    edge = np.zeros((h, w), np.uint8)
+    lib().orc_sample_draft_tokens(C.byref(params), _ptr(np.ascontiguousarray(draft_lo)), _ptr(tok), _ptr(edge))
+    return (tok, edge) if with_edge else tok
+
+
+def downsample_majority(x, r):
+    """Step 7 stand-in: the most frequent token of every r x r block (ties: first in raster order)."""
+    x = np.ascontiguousarray(x, np.int32)
+    H, W = x.shape
+    y = np.empty((H // r, W // r), np.int32)
+    lib().orc_downsample_majority(_ptr(x), H, W, int(r), _ptr(y))
+    return y
 
 
 # --------------------------------------------------------------------- stages

@@ -20,6 +20,8 @@
  *   Sec. 3.3 Eq. 7   R_X = union of N(t,l) over rejected t
  *   Algorithm 1      Step 4 (accept), Step 5 (expand), Step 6 (resample from M_p)
  *   Sec. 3.4 Eq. 8   rejection islands {I_m} = CC_8(R_X): 8-connected components
+ *   Sec. 3.2 Step 1  y~ ~ M_q: the drafter's own sampling, on given logits
+ *   Sec. 3.2 Step 7  y = D_r(x): stand-in, majority token of each r x r block
  *   Supp. "Sampling" temperature, top-k, classifier-free guidance of the sampler
  *
  * Readings taken where the paper is silent (each is listed in the design notes):
@@ -50,7 +52,10 @@
  * chi-square of the whole round; dilation against scipy and brute force;
  * inverse CDF against numpy.searchsorted; islands against scipy.ndimage.label,
  * against reachability by boolean matrix closure on every mask of a small grid,
- * and on hand-drawn shapes.  The paper prints no worked numeric example for this
+ * and on hand-drawn shapes; the draft sampler against the pinned primitives
+ * composed in the test and by chi-square over rounds; the down-sampler by
+ * D_r(U_r(y)) = y, scipy.stats.mode on blocks without ties, and hand-written
+ * blocks with ties.  The paper prints no worked numeric example for this
  * path, so no pin is a printed value.
  */
 #include <math.h>
@@ -574,22 +579,49 @@ void orc_inverse_cdf_histogram(const double* w, int V, uint32_t n_begin, uint32_
   }
 }
 
-/* Draw one token per low-res cell from q (after temperature / top-k) with the
- * tag-1 Philox stream: the draft model's own sampling (Step 1), used only to
- * make inputs for the CPU pins. */
-void orc_sample_draft_tokens(const orc_params* P, const void* draft_lo, int32_t* draft_tok_lo) {
+/* Step 1 on given logits: one token per low-res cell from q (after temperature /
+ * top-k) by inverse CDF in ascending token id, uniform = word 0 of the tag-1
+ * Philox stream at (cell, image, round).  edge[cell] (may be NULL) = 1 where the
+ * uniform lies within 1e-6 of an edge of the chosen CDF bin. */
+void orc_sample_draft_tokens(const orc_params* P, const void* draft_lo, int32_t* draft_tok_lo,
+                             uint8_t* edge) {
   const int V = P->V, h = P->H / P->r, w = P->W / P->r;
   const size_t esz = P->dtype == ORC_BF16 ? 2 : 4;
   float* z = (float*)malloc((size_t)V * sizeof(float));
   double* q = (double*)malloc((size_t)V * sizeof(double));
   for (int cell = 0; cell < h * w; ++cell) {
-    double m, Z, u[3];
+    double m, Z, u[3], gap;
     orc_preprocess_row((const char*)draft_lo + (size_t)cell * V * esz, NULL, P->dtype, V, 0.0f,
                        P->temperature, z);
     orc_softmax_masked(z, V, orc_topk_threshold(z, V, P->top_k), q, &m, &Z);
     orc_position_uniforms(P->seed, P->image, (uint32_t)cell, P->round, 1u, u);
-    draft_tok_lo[cell] = orc_inverse_cdf(q, V, u[0], NULL, NULL);
+    draft_tok_lo[cell] = orc_inverse_cdf(q, V, u[0], NULL, &gap);
+    if (edge) edge[cell] = gap < 1e-6;
   }
   free(z);
   free(q);
+}
+
+/* Step 7 stand-in.  The paper's D_r is a trained network; the stand-in keeps the
+ * one property the round relies on, D_r(U_r(y)) = y for the replicating U_r:
+ * y[a][c] is the token that occurs most often among the r x r tokens
+ * x[a r + di][c r + dj]; among tokens with the same count, the one that occurs
+ * first in raster order of the block. */
+void orc_downsample_majority(const int32_t* x, int H, int W, int r, int32_t* y) {
+  const int h = H / r, w = W / r;
+  for (int a = 0; a < h; ++a)
+    for (int c = 0; c < w; ++c) {
+      int best_tok = -1, best_count = 0;
+      for (int s = 0; s < r * r; ++s) {
+        const int tok = x[(a * r + s / r) * W + c * r + s % r];
+        int count = 0;
+        for (int s2 = 0; s2 < r * r; ++s2)
+          if (x[(a * r + s2 / r) * W + c * r + s2 % r] == tok) ++count;
+        if (count > best_count) { /* strict: an earlier token keeps a tie */
+          best_count = count;
+          best_tok = tok;
+        }
+      }
+      y[a * w + c] = best_tok;
+    }
 }
