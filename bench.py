@@ -468,6 +468,82 @@ def run_islands(args, cfg):
     ctx.close()
 
 
+def run_draft_io(args, cfg):
+    """Step 1 (the drafter's own sampling on given logits) and the Step 7 stand-in (majority down-sampler) on
+    the workload's shapes: one JSON line each, with the CPU oracle timed on a bounded sample.  Single GPU."""
+    from paper_2601_05149_b200 import binding
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: these stages have no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    ctx = binding.Context(0)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else 6650.0
+    batch = synth.build_batch(cfg, dev)
+    p = binding.params_from_config(cfg)
+    ctx.ensure_workspace(p)
+    W, K = max(3, args.warmup), max(1, args.steps)
+    esz = 2 if cfg.dtype == "bf16" else 4
+    cells = cfg.B * cfg.h * cfg.w
+    tok_lo = torch.empty((cfg.B, cfg.h, cfg.w), dtype=torch.int32, device=dev)
+    tok_hi = torch.randint(0, cfg.V, (cfg.B, cfg.H, cfg.W), dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+
+    def timed(fn):
+        e = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for s_ in range(W + K):
+            flush.zero_()
+            p.round = s_
+            if s_ >= W:
+                e[s_ - W][0].record()
+            fn()
+            if s_ >= W:
+                e[s_ - W][1].record()
+        torch.cuda.synchronize()
+        return statistics.mean(a.elapsed_time(b) for a, b in e)
+
+    def line(stage, kernel, metric, units, ms, alg, cpu):
+        print(json.dumps({
+            "stage": stage, "metric": metric, "value": units / (ms * 1e-3), "unit": metric.split("_per_")[0] + "/s",
+            "ms_per_step": ms, "steps": K, "warmup": W, "dtype": "f32" if stage == "mulo_sample_draft" else "int32",
+            "data": "synthetic",
+            "config": {"workload": workload_desc(cfg), "l2": "256 MB written between timed launches"},
+            "roofline": {"bound": "hbm", "kernel": kernel, "achieved": alg / (ms * 1e-3) / 1e9, "peak": peak,
+                         "unit": "GB/s", "frac": alg / (ms * 1e-3) / 1e9 / peak, "bytes_per_launch": alg,
+                         "traffic": None},
+            "cpu_baseline": cpu}), flush=True)
+
+    import oracle
+
+    def orc_params(b):
+        return oracle.make_params(cfg.H, cfg.W, cfg.V, cfg.r, oracle.BF16 if cfg.dtype == "bf16" else oracle.F32,
+                                  temperature=cfg.temperature, top_k=cfg.top_k, seed=cfg.seed, round=0, image=b)
+    ms = timed(lambda: ctx.mulo_sample_draft(p, batch["draft_lo"], tok_lo))
+    cpu = None
+    if not args.no_cpu_baseline:
+        n_img = min(cfg.B, 2)
+        t0 = time.time()
+        for b in range(n_img):
+            oracle.sample_draft_tokens(orc_params(b), synth.to_numpy_logits(batch["draft_lo"][b]))
+        dt = time.time() - t0
+        cpu = {"value": n_img * cfg.h * cfg.w / dt, "unit": "cells/s", "cores": 1, "kind": "oracle",
+               "sample": f"{n_img} of {cfg.B} images", "seconds": dt}
+    line("mulo_sample_draft", "k_sample_draft", "cells_per_sec", cells, ms, cells * (cfg.V * esz + 4), cpu)
+
+    ms = timed(lambda: ctx.mulo_downsample(p, tok_hi, tok_lo))
+    cpu = None
+    if not args.no_cpu_baseline:
+        x = tok_hi.cpu().numpy()
+        t0 = time.time()
+        for b in range(cfg.B):
+            oracle.downsample_majority(x[b], cfg.r)
+        dt = time.time() - t0
+        cpu = {"value": cells / dt, "unit": "cells/s", "cores": 1, "kind": "oracle",
+               "sample": f"all {cfg.B} images", "seconds": dt}
+    line("mulo_downsample", "k_downsample", "cells_per_sec", cells, ms, cells * 4 * (cfg.r * cfg.r + 1), cpu)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -481,6 +557,8 @@ def main():
     ap.add_argument("--sweep-limit", type=int, default=0, help="only the first N sweep points")
     ap.add_argument("--islands", action="store_true",
                     help="time the rejection-island labelling of the workload's masks instead of the bench line")
+    ap.add_argument("--draft-io", action="store_true",
+                    help="time the drafter's sampling and the down-sampler stand-in instead of the bench line")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.workload]
     if args.batch:
@@ -489,6 +567,8 @@ def main():
         run_sweep(args)
     elif args.islands:
         run_islands(args, cfg)
+    elif args.draft_io:
+        run_draft_io(args, cfg)
     elif args.impl == "reference":
         run_reference(args, cfg)
     else:

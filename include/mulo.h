@@ -192,6 +192,24 @@ mulo_status mulo_local_reject_expand(mulo_ctx* ctx, const mulo_params* p,
                                      const uint32_t* reject_bits, const int32_t* first_reject,
                                      uint32_t* expand_bits, int32_t* n_expand, void* stream);
 
+/* Step 1 on given logits (Sec. 3.2): the drafter's own draw y~ ~ q, one token per low-res cell,
+ * by inverse CDF in ascending token id over q = softmax(topk(l_q / T)) (same temperature and
+ * top-k as the round).  The uniform is word 0 of the Philox stream with counter
+ * (cell index a * w + c, image b + image_offset, round, 1): the last counter word tells it
+ * apart from the round's own uniforms, which use 0 there.  Needs a workspace (status word).
+ *   draft_logits_lo [B, h, w, V]  in      draft_tok_lo [B, h, w]  out                       */
+mulo_status mulo_sample_draft(mulo_ctx* ctx, const mulo_params* p, const void* draft_logits_lo,
+                              int32_t* draft_tok_lo, void* stream);
+
+/* Step 7 stand-in (Sec. 3.2: y = D_r(x), the prefix of the next low-resolution draft).  The
+ * paper's D_r is a trained network; this call keeps the one property the round relies on,
+ * D_r(U_r(y)) = y for the replicating up-sampler: tok_lo[a][c] is the token that occurs most
+ * often in the r x r block tok_hi[a r .. a r + r - 1][c r .. c r + r - 1]; among tokens with
+ * the same count, the one that comes first in raster order of the block.  r <= 16.
+ *   tok_hi [B, H, W]  in      tok_lo [B, h, w]  out                                          */
+mulo_status mulo_downsample(mulo_ctx* ctx, const mulo_params* p, const int32_t* tok_hi,
+                            int32_t* tok_lo, void* stream);
+
 /* Rejection islands (Sec. 3.4, Eq. 8): {I_m} = CC_8(R_X), the 8-connected components of R_X
  * on the token grid (two positions are neighbours when both coordinates differ by at most
  * one), which a scheduler redraws concurrently.  Uses B, H, W of `p`; H * W <= 16384, else

@@ -99,6 +99,46 @@ __global__ void __launch_bounds__(kThreads) k_upsample_pool(RowKernelArgs a) {
   }
 }
 
+// mulo_sample_draft: one CTA per low-res cell; the drafter's own draw (Sec. 3.2 Step 1) from
+// q = softmax(topk(l_q / T)) with word 0 of the tag-1 Philox stream.
+__global__ void __launch_bounds__(kThreads) k_sample_draft(RowKernelArgs a) {
+  __shared__ BlockScratch bs;
+  const DevParams& P = a.P;
+  const int cell = blockIdx.x;   // b*h*w + ca*w + cc
+  const int b = cell / (P.h * P.w), rem = cell % (P.h * P.w);
+  RowSrc qr = draft_row(a, cell);
+  RowStats sq;
+  dense_row_stats(qr, P.top_k, bs, sq.theta, sq.m, sq.Z);
+  __syncthreads();
+  const float invZ = (float)(1.0 / sq.Z);
+  const uint4 rnd = philox4x32_10(make_uint4((uint32_t)rem, (uint32_t)b + P.image_offset, P.round, 1u),
+                                  make_uint2(P.seed_lo, P.seed_hi));
+  // lambda = 0 and no special token: the weights are q itself
+  const int tok = dense_draw(qr, qr, sq, sq, invZ, invZ, 0.0f, -1, 0.0, nullptr, uniform24(rnd.x), bs);
+  if (threadIdx.x == 0) a.out_tok[cell] = tok;
+}
+
+// mulo_downsample: one thread per low-res cell; the most frequent token of its r x r block,
+// ties to the one that comes first in raster order of the block (Step 7 stand-in).
+__global__ void __launch_bounds__(256) k_downsample(const int32_t* __restrict__ x, int32_t* __restrict__ y,
+                                                    int cells, int h, int w, int W, int r) {
+  const int cell = blockIdx.x * blockDim.x + threadIdx.x;
+  if (cell >= cells) return;
+  const int b = cell / (h * w), rem = cell % (h * w), ca = rem / w, cc = rem % w;
+  const int32_t* blk = x + ((size_t)b * h * r + (size_t)ca * r) * W + (size_t)cc * r;
+  int best_tok = -1, best_count = 0;
+  for (int s1 = 0; s1 < r * r; ++s1) {
+    const int tok = blk[(size_t)(s1 / r) * W + s1 % r];
+    int count = 0;
+    for (int s2 = 0; s2 < r * r; ++s2) count += blk[(size_t)(s2 / r) * W + s2 % r] == tok;
+    if (count > best_count) {
+      best_count = count;
+      best_tok = tok;
+    }
+  }
+  y[cell] = best_tok;
+}
+
 // mulo_verify (FUSED = false): one CTA per target position, draft statistics given.
 // mulo_round  (FUSED = true):  one CTA per low-res cell: draft statistics, then its
 // r*r children; accept flags and candidate draws go to the workspace.
@@ -722,6 +762,37 @@ mulo_status mulo_upsample_pool(mulo_ctx* ctx, const mulo_params* p, const void* 
   a.q_tok_hi_out = q_tok_hi;
   a.dev_status = (uint32_t*)ctx->ws;
   k_upsample_pool<<<p->B * a.P.h * a.P.w, kThreads, 0, (cudaStream_t)stream>>>(a);
+  return launched(ctx, 1);
+}
+
+mulo_status mulo_sample_draft(mulo_ctx* ctx, const mulo_params* p, const void* draft_logits_lo,
+                              int32_t* draft_tok_lo, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!draft_logits_lo || !draft_tok_lo || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
+  if (!ctx->ws) return MULO_ERR_WORKSPACE;
+  if (p->B == 0) return MULO_OK;
+  RowKernelArgs a;
+  memset(&a, 0, sizeof a);
+  a.P = to_dev(p);
+  a.draft = (const char*)draft_logits_lo;
+  a.out_tok = draft_tok_lo;
+  a.dev_status = (uint32_t*)ctx->ws;
+  k_sample_draft<<<p->B * a.P.h * a.P.w, kThreads, 0, (cudaStream_t)stream>>>(a);
+  return launched(ctx, 1);
+}
+
+mulo_status mulo_downsample(mulo_ctx* ctx, const mulo_params* p, const int32_t* tok_hi, int32_t* tok_lo,
+                            void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!tok_hi || !tok_lo) return MULO_ERR_INVALID_ARG;
+  if (p->r > 16) return MULO_ERR_UNSUPPORTED;
+  if (p->B == 0) return MULO_OK;
+  const int h = p->H / p->r, w = p->W / p->r, cells = p->B * h * w;
+  k_downsample<<<(cells + 255) / 256, 256, 0, (cudaStream_t)stream>>>(tok_hi, tok_lo, cells, h, w, p->W, p->r);
   return launched(ctx, 1);
 }
 
