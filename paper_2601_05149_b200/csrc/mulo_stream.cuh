@@ -377,30 +377,50 @@ __device__ __forceinline__ int warp_draw(const float* seg, int n_seg, const usho
   if (!(total > 0.0)) return -1;
   const double y = u * total;
   const unsigned hit = __ballot_sync(kFull, loc > 0.0 && inc > y);
-  if (hit) {
-    const int l = __ffs(hit) - 1;
-    double acc = __shfl_sync(kFull, inc - loc, l);   // mass before lane l's block
-    for (int i = 0; i < per; ++i) {                  // the same walk in every lane
-      const int sidx = l * per + i;
-      if (sidx >= n_seg) break;
-      const double w = (double)seg[sidx];
-      if (w > 0.0 && acc + w > y) {
-        const ushort2 r = run[sidx];
-        const int at = warp_locate((int)r.y, (float)(y - acc), [&](int k) { return wfun((int)r.x + k); });
-        if (at >= 0) return (int)r.x + at;
+  // Segments to try, the same in every lane: forward through the block of the lane that holds
+  // u * total; then, should rounding have left u * total at (or past) the end, backward from
+  // the last segment for the last entry with weight.  One call site for the search inside a
+  // segment keeps the code small.
+  const int l = hit ? __ffs(hit) - 1 : 0;
+  double acc = __shfl_sync(kFull, inc - loc, l);   // mass before lane l's block
+  int sidx = hit ? l * per : n_seg - 1;
+  const int fwd_end = min((l + 1) * per, n_seg);
+  bool forward = hit != 0;
+#pragma unroll 1
+  for (;;) {
+    float yy;
+    double w = 0.0;
+    if (forward) {
+      if (sidx >= fwd_end) {
+        forward = false;
+        sidx = n_seg - 1;
+        continue;
       }
+      w = (double)seg[sidx];
+      if (!(w > 0.0 && acc + w > y)) {
+        acc += w;
+        ++sidx;
+        continue;
+      }
+      yy = (float)(y - acc);
+    } else {
+      if (sidx < 0) return -1;
+      if (!(seg[sidx] > 0.f)) {
+        --sidx;
+        continue;
+      }
+      yy = 3.0e38f;
+    }
+    const ushort2 r = run[sidx];
+    const int at = warp_locate((int)r.y, yy, [&](int k) { return wfun((int)r.x + k); });
+    if (at >= 0) return (int)r.x + at;
+    if (forward) {
       acc += w;
+      ++sidx;
+    } else {
+      --sidx;
     }
   }
-  // rounding left u * total at (or past) the end: the last entry with weight
-  for (int sidx = n_seg - 1; sidx >= 0; --sidx) {
-    if (seg[sidx] > 0.f) {
-      const ushort2 r = run[sidx];
-      const int at = warp_locate((int)r.y, 3.0e38f, [&](int k) { return wfun((int)r.x + k); });
-      if (at >= 0) return (int)r.x + at;
-    }
-  }
-  return -1;
 }
 
 // where the k-th largest value lies in a row's selection histogram
@@ -1135,24 +1155,27 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         }
         __syncthreads();
         reset_state();
-        if (ok) {
-          if (warp == 0) {
-            int t_res = -1;
-            if (draws & kDrawResidual) {
-              int at = warp_draw(seg_b, a.n_seg, tseg, uniform24(pp.rnd[1]), w_resid);
-              if (at < 0)   // residual without mass: the target weights, same uniform
-                at = warp_draw(seg_c, a.n_seg, tseg, uniform24(pp.rnd[1]), w_target);
-              t_res = at >= 0 ? (int)cand[at].y : -1;
+        if (ok && warp < 2) {
+          // warp 0: the draw from the residual (a residual without mass falls back to the target
+          // weights with the same uniform); warp 1: the draw from the target distribution.  Both
+          // run the same code, the weight function picked at run time.
+          int t_out = -1;
+          if (draws & (warp == 0 ? kDrawResidual : kDrawTarget)) {
+            bool resid = warp == 0;
+            const double u = uniform24(pp.rnd[warp == 0 ? 1 : 2]);
+#pragma unroll 1
+            for (int attempt = 0; attempt < 2; ++attempt) {
+              const int at = warp_draw(resid ? seg_b : seg_c, a.n_seg, tseg, u,
+                                       [&](int i) { return resid ? w_resid(i) : w_target(i); });
+              if (at >= 0) {
+                t_out = (int)cand[at].y;
+                break;
+              }
+              if (!resid) break;
+              resid = false;
             }
-            if (lane == 0) a.cand_res[g] = t_res;
-          } else if (warp == 1) {
-            int t_tgt = -1;
-            if (draws & kDrawTarget) {
-              const int at = warp_draw(seg_c, a.n_seg, tseg, uniform24(pp.rnd[2]), w_target);
-              t_tgt = at >= 0 ? (int)cand[at].y : -1;
-            }
-            if (lane == 0) a.cand_tgt[g] = t_tgt;
           }
+          if (lane == 0) (warp == 0 ? a.cand_res : a.cand_tgt)[g] = t_out;
         }
         if ((tid == 64 || tid == 96) && child + 1 < rr) prepare_row(sm.prep[(rowi + 1) & 1], child + 1, tid == 96);
         if (tid == 128) learn(1, ok_sel, s.reason, theta, pivot, s.n, n_ge);
