@@ -528,7 +528,7 @@ def run_draft_io(args, cfg):
         dt = time.time() - t0
         cpu = {"value": n_img * cfg.h * cfg.w / dt, "unit": "cells/s", "cores": 1, "kind": "oracle",
                "sample": f"{n_img} of {cfg.B} images", "seconds": dt}
-    line("mulo_sample_draft", "k_sample_draft", "cells_per_sec", cells, ms, cells * (cfg.V * esz + 4), cpu)
+    line("mulo_sample_draft", "k_round_stream<sampling mode> (+ k_sample_failed)", "cells_per_sec", cells, ms, cells * (cfg.V * esz + 4), cpu)
 
     ms = timed(lambda: ctx.mulo_downsample(p, tok_hi, tok_lo))
     cpu = None

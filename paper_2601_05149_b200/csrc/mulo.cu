@@ -99,12 +99,10 @@ __global__ void __launch_bounds__(kThreads) k_upsample_pool(RowKernelArgs a) {
   }
 }
 
-// mulo_sample_draft: one CTA per low-res cell; the drafter's own draw (Sec. 3.2 Step 1) from
-// q = softmax(topk(l_q / T)) with word 0 of the tag-1 Philox stream.
-__global__ void __launch_bounds__(kThreads) k_sample_draft(RowKernelArgs a) {
-  __shared__ BlockScratch bs;
+// The drafter's own draw (Sec. 3.2 Step 1) for one low-res cell by the general routines:
+// q = softmax(topk(l_q / T)), inverse CDF with word 0 of the tag-1 Philox stream.
+__device__ inline void sample_cell(const RowKernelArgs& a, int cell, BlockScratch& bs) {
   const DevParams& P = a.P;
-  const int cell = blockIdx.x;   // b*h*w + ca*w + cc
   const int b = cell / (P.h * P.w), rem = cell % (P.h * P.w);
   RowSrc qr = draft_row(a, cell);
   RowStats sq;
@@ -116,6 +114,25 @@ __global__ void __launch_bounds__(kThreads) k_sample_draft(RowKernelArgs a) {
   // lambda = 0 and no special token: the weights are q itself
   const int tok = dense_draw(qr, qr, sq, sq, invZ, invZ, 0.0f, -1, 0.0, nullptr, uniform24(rnd.x), bs);
   if (threadIdx.x == 0) a.out_tok[cell] = tok;
+}
+
+// mulo_sample_draft, general path: one CTA per low-res cell.
+__global__ void __launch_bounds__(kThreads) k_sample_draft(RowKernelArgs a) {
+  __shared__ BlockScratch bs;
+  sample_cell(a, blockIdx.x, bs);
+}
+
+// Second launch of mulo_sample_draft's fast path: the cells the streaming kernel put on its list.
+__global__ void __launch_bounds__(kThreads) k_sample_failed(RowKernelArgs a, const int32_t* fail_list,
+                                                            const uint32_t* fail_count) {
+  __shared__ BlockScratch bs;
+  const size_t total = (size_t)a.P.B * a.P.h * a.P.w;
+  const size_t n = min((size_t)*fail_count, total);
+  for (size_t idx = blockIdx.x; idx < n; idx += gridDim.x) {
+    const size_t cell = (size_t)fail_list[idx];
+    if (cell < total) sample_cell(a, (int)cell, bs);
+    __syncthreads();
+  }
 }
 
 // mulo_downsample: one thread per low-res cell; the most frequent token of its r x r block,
@@ -713,9 +730,9 @@ static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s
   return dyn;
 }
 
-template <bool BF16, bool HAS_U>
+template <bool BF16, bool HAS_U, bool SAMPLE = false>
 static bool launch_stream_t(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn, cudaStream_t st) {
-  auto kern = k_round_stream<BF16, HAS_U>;
+  auto kern = k_round_stream<BF16, HAS_U, SAMPLE>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
     cudaGetLastError();
     return false;
@@ -773,13 +790,35 @@ mulo_status mulo_sample_draft(mulo_ctx* ctx, const mulo_params* p, const void* d
   if (!draft_logits_lo || !draft_tok_lo || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
   if (!ctx->ws) return MULO_ERR_WORKSPACE;
   if (p->B == 0) return MULO_OK;
+  cudaStream_t st = (cudaStream_t)stream;
   RowKernelArgs a;
   memset(&a, 0, sizeof a);
   a.P = to_dev(p);
   a.draft = (const char*)draft_logits_lo;
   a.out_tok = draft_tok_lo;
   a.dev_status = (uint32_t*)ctx->ws;
-  k_sample_draft<<<p->B * a.P.h * a.P.w, kThreads, 0, (cudaStream_t)stream>>>(a);
+  // fast path: the streaming kernel in its sampling mode (top-k on, and a workspace large
+  // enough for the list of cells it may leave to the general routines)
+  Workspace w;
+  StreamArgs sa;
+  memset(&sa, 0, sizeof sa);
+  const size_t sdyn = (ctx->force_dense || check_ws(ctx, p, &w) != MULO_OK) ? 0 : plan_stream(ctx, a.P, &sa);
+  if (sdyn) {
+    sa.P = a.P;
+    sa.draft = a.draft;
+    sa.sample_out = draft_tok_lo;
+    sa.dev_status = w.status;
+    sa.fail_list = w.fail_list;
+    sa.n_parents = p->B * a.P.h * a.P.w;
+    if (cudaMemsetAsync(w.status + kFailCount, 0, sizeof(uint32_t), st) != cudaSuccess) return MULO_ERR_CUDA;
+    const bool fast = a.P.bf16 ? launch_stream_t<true, false, true>(ctx, sa, sdyn, st)
+                               : launch_stream_t<false, false, true>(ctx, sa, sdyn, st);
+    if (fast) {
+      k_sample_failed<<<2 * ctx->sm_count, kThreads, 0, st>>>(a, w.fail_list, w.status + kFailCount);
+      return launched(ctx, 2);
+    }
+  }
+  k_sample_draft<<<p->B * a.P.h * a.P.w, kThreads, 0, st>>>(a);
   return launched(ctx, 1);
 }
 

@@ -133,6 +133,7 @@ struct StreamArgs {
   const char* uncond;
   const char* draft;
   const int32_t* draft_tok_lo;
+  int32_t* sample_out;   // sampling mode: [B, h, w] the drafter's own draw per low-res cell
   float* p_tok;
   float* q_tok;
   float* accept_prob;
@@ -359,7 +360,8 @@ __device__ __forceinline__ int warp_locate(int cnt, float y, W wfun) {
 // segment that holds u * total, then the entry inside it.  Returns the index into
 // the candidate array, or -1 when the total is zero.  Call from all lanes of ONE warp.
 template <class W>
-__device__ __forceinline__ int warp_draw(const float* seg, int n_seg, const ushort2* run, double u, W wfun) {
+__device__ __forceinline__ int warp_draw(const float* seg, int n_seg, const ushort2* run, double u, W wfun,
+                                         int* seg_out = nullptr) {
   const int lane = threadIdx.x & 31;
   // every lane sums a block of consecutive segments, then one scan over the lanes
   const int per = (n_seg + 31) / 32;
@@ -413,7 +415,10 @@ __device__ __forceinline__ int warp_draw(const float* seg, int n_seg, const usho
     }
     const ushort2 r = run[sidx];
     const int at = warp_locate((int)r.y, yy, [&](int k) { return wfun((int)r.x + k); });
-    if (at >= 0) return (int)r.x + at;
+    if (at >= 0) {
+      if (seg_out) *seg_out = sidx;
+      return (int)r.x + at;
+    }
     if (forward) {
       acc += w;
       ++sidx;
@@ -434,8 +439,12 @@ struct Sel {
                 // 3 k-th largest above the histogram, 4 too many ties at the threshold
 };
 
-template <bool BF16, bool HAS_U>
+// SAMPLE = true turns the kernel into the drafter's own sampling (Sec. 3.2 Step 1): only the draft
+// rows are streamed (one row per "parent"), and instead of verifying children one warp draws
+// y~ ~ q from the row's candidate list with word 0 of the tag-1 Philox stream.
+template <bool BF16, bool HAS_U, bool SAMPLE = false>
 __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_constant__ StreamArgs a) {
+  static_assert(!(SAMPLE && HAS_U), "draft rows have no unconditional stream");
   constexpr int EPL = BF16 ? 8 : 4;        // entries per lane visit (16 bytes of the conditional row)
   constexpr int PIECE = 32 * EPL;          // entries per 32-lane piece
   constexpr int SEG = kPPW * PIECE;        // entries of the row that one segment covers
@@ -464,7 +473,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
   const int p_begin = (int)(((long long)a.n_parents * blockIdx.x) / gridDim.x);
   const int p_end = (int)(((long long)a.n_parents * (blockIdx.x + 1)) / gridDim.x);
   if (p_end <= p_begin) return;
-  const int rr = P.r * P.r, rows_per_parent = 1 + rr;
+  const int rr = SAMPLE ? 0 : P.r * P.r, rows_per_parent = 1 + rr;
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -849,7 +858,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       acc = seg_lanes_sum(acc, seg_lanes);
       if (sub == 0 && has) {
         seg_a[seg] = acc;
-        if (!IS_Q) seg_c[seg] = acc;
+        if (!IS_Q || SAMPLE) seg_c[seg] = acc;
       }
     }
   };
@@ -892,7 +901,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       if (keep) {
         const float e = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
         z += (double)e;
-        if (own && !IS_Q) atomicAdd(&seg_c[seg], e);
+        if (own && (!IS_Q || SAMPLE)) atomicAdd(&seg_c[seg], e);
       } else if (own) {
         if (IS_Q) qval[at] = 0.f;
         else cand[at].x = 0u;
@@ -995,7 +1004,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     // ------------------------------------------------------------ draft row
     {
       if (tid == 0) {
-        sm.tok = checked_token(a.draft_tok_lo[parent], P.V, a.dev_status);
+        if (!SAMPLE) sm.tok = checked_token(a.draft_tok_lo[parent], P.V, a.dev_status);
         // row addresses two parents ahead
         const int tp = sm.tparent + 1;
         if (parent > p_begin && tp < p_end) {
@@ -1018,7 +1027,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       choose_pivot(0, std::false_type{}, pivot, inv_w);
       stream_row(std::true_type{}, std::false_type{}, pivot, inv_w);
       __syncthreads();
-      if (tid == 64) prefetch_row(0);
+      if (!SAMPLE && tid == 64) prefetch_row(0);
       Sel s;
       bool ok = locate_bin(s);
       float theta = 0.f;
@@ -1030,7 +1039,12 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       if (tid == 0) {
         learn(0, ok, s.reason, theta, pivot, s.n, n_ge);
         sm.q_ok = ok;
-        if (ok) {
+        if (SAMPLE) {
+          if (!ok) {
+            atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
+            defer((size_t)parent);
+          }
+        } else if (ok) {
           // same rounding of Z_q as the unfused path (fp32 hi + lo)
           const float Zhi = (float)Zq, Zlo = (float)(Zq - (double)Zhi);
           const double Z = (double)Zhi + (double)Zlo;
@@ -1051,8 +1065,46 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       }
       __syncthreads();   // everybody is done with the selection scratch
       reset_state();
-      if ((tid == 64 || tid == 96) && ok) prepare_row(sm.prep[rowi & 1], 0, tid == 96);   // first child's uniforms and logit of x~
+      if (!SAMPLE && (tid == 64 || tid == 96) && ok)
+        prepare_row(sm.prep[rowi & 1], 0, tid == 96);   // first child's uniforms and logit of x~
+      if (SAMPLE && ok && warp == 0) {
+        // y~ ~ q: inverse CDF over the row's candidate list (e = 0 below theta_q), then the token
+        // id of the chosen entry from the look-up table of its segment
+        const uint4 rnd = philox4x32_10(
+            make_uint4((uint32_t)(sm.ca * P.w + sm.cc), (uint32_t)sm.b + P.image_offset, P.round, 1u),
+            make_uint2(P.seed_lo, P.seed_hi));
+        int sidx = 0;
+        const int at = warp_draw(seg_c, a.n_seg, qseg, uniform24(rnd.x), [&](int i) { return qval[i]; }, &sidx);
+        int tok = -1;
+        if (at >= 0) {
+          const int local = at - (int)qseg[sidx].x;   // rank of the entry within its segment
+          const int cell0 = ((sidx / kSWarps) * a.chunk + (sidx % kSWarps) * SEG) / EPL;
+          int found = -1;
+          for (int k = lane; k < SEG / EPL; k += 32) {
+            const unsigned cell = (cell0 + k) * EPL < P.V ? qcell[cell0 + k] : 0u;
+            const unsigned m8 = cell & 0xffu;
+            const int off = (int)(cell >> 8);
+            if (m8 && off <= local && local < off + __popc(m8))
+              found = (cell0 + k) * EPL + (int)__fns(m8, 0, local - off + 1);
+          }
+          const unsigned who = __ballot_sync(kFull, found >= 0);
+          if (who) tok = __shfl_sync(kFull, found, __ffs(who) - 1);
+        }
+        if (lane == 0) a.sample_out[parent] = tok;
+      }
       __syncthreads();
+    }
+    if (SAMPLE) {
+      if (tid == 0) {   // next cell's coordinates (made visible by the barriers of its row)
+        if (++sm.cc == P.w) {
+          sm.cc = 0;
+          if (++sm.ca == P.h) {
+            sm.ca = 0;
+            ++sm.b;
+          }
+        }
+      }
+      continue;
     }
 
     // ------------------------------------------------------------ children

@@ -62,6 +62,51 @@ def test_sample_draft_small(ctx, cfg):
     sample_both(ctx, cfg)
 
 
+@pytest.mark.parametrize("cfg", [
+    dataclasses.replace(TINY, B=2, H=16, W=16, V=16384, dtype="bf16", top_k=2000, seed=330),
+    dataclasses.replace(TINY, B=2, H=16, W=16, V=4096, dtype="f32", top_k=500, temperature=0.8, seed=331),
+    dataclasses.replace(TINY, B=1, H=8, W=8, V=4104, dtype="bf16", top_k=300, seed=332),     # ragged last chunk
+    dataclasses.replace(TINY, B=1, H=8, W=8, V=65536, dtype="bf16", top_k=4000, seed=333),   # sixteen chunks per row
+], ids=lambda c: f"{c.dtype}-V{c.V}-k{c.top_k}")
+def test_sample_draft_fast_path(ctx, cfg):
+    """Top-k on and V >= 1024: the streaming kernel in its sampling mode (two launches), same parity bar;
+    switched off, the general kernel (one launch) meets it too."""
+    ctx.ensure_workspace(binding.params_from_config(cfg))
+    n0 = ctx.kernel_launches()
+    sample_both(ctx, cfg)
+    assert ctx.kernel_launches() - n0 == 2
+    lost = ctx.poll_fallback_counts()[0]
+    assert lost <= cfg.B * cfg.h * cfg.w // 4
+    ctx.set_general_path_only(True)
+    try:
+        n0 = ctx.kernel_launches()
+        sample_both(ctx, cfg)
+        assert ctx.kernel_launches() - n0 == 1
+    finally:
+        ctx.set_general_path_only(False)
+
+
+def test_sample_draft_fast_path_rows_that_are_not_normal(ctx):
+    """Heavy-tailed rows defeat the pivot prediction now and then: those cells go through the list."""
+    cfg = dataclasses.replace(TINY, B=2, H=32, W=32, V=4096, dtype="f32", top_k=400, seed=334)
+    batch = pu.build_batch(cfg)
+    batch["draft_lo"] = (batch["draft_lo"] ** 3).contiguous()
+    p = binding.params_from_config(cfg)
+    ctx.ensure_workspace(p)
+    tok = torch.full((cfg.B, cfg.h, cfg.w), -5, dtype=torch.int32, device="cuda")
+    ctx.mulo_sample_draft(p, batch["draft_lo"], tok)
+    torch.cuda.synchronize()
+    tok = tok.cpu().numpy()
+    differ = 0
+    for b in range(cfg.B):
+        want, edge = oracle.sample_draft_tokens(pu.orc_params(cfg, b), synth.to_numpy_logits(batch["draft_lo"][b]),
+                                                with_edge=True)
+        bad = (tok[b] != want) & (edge == 0)
+        assert not bad.any(), (b, np.argwhere(bad)[:5])
+        differ += int((tok[b] != want).sum())
+    assert differ <= 2
+
+
 def test_sample_draft_streams(ctx):
     """Different rounds and image offsets draw different tokens; the same ones repeat exactly."""
     cfg = dataclasses.replace(TINY, B=2, dtype="bf16", top_k=40, seed=310)
