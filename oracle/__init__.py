@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
             _lib.orc_inverse_cdf.restype = C.c_int
             _lib.orc_expand.restype = C.c_int
             _lib.orc_islands.restype = C.c_int
+            _lib.orc_island_schedule.restype = C.c_int
     return _lib
 
 
@@ -192,6 +193,16 @@ def islands(in_rx):
     size = np.zeros(max(H * W, 1), np.int32)
     M = int(lib().orc_islands(_ptr(in_rx), H, W, _ptr(labels), _ptr(rows), _ptr(size)))
     return labels, M, rows[:M].copy(), size[:M].copy()
+
+
+def island_schedule(labels, window):
+    """Step index of every position of R_X under the row-window rule (0 outside R_X) and the number of
+    sequential steps of the image."""
+    labels = np.ascontiguousarray(labels, np.int32)
+    H, W = labels.shape
+    step = np.zeros((H, W), np.int32)
+    nfe = int(lib().orc_island_schedule(_ptr(labels), H, W, int(window), _ptr(step)))
+    return step, nfe
 
 
 def position_distributions(params, cond_row, uncond_row, draft_row, tok, nn=None):

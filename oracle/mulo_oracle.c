@@ -20,6 +20,7 @@
  *   Sec. 3.3 Eq. 7   R_X = union of N(t,l) over rejected t
  *   Algorithm 1      Step 4 (accept), Step 5 (expand), Step 6 (resample from M_p)
  *   Sec. 3.4 Eq. 8   rejection islands {I_m} = CC_8(R_X): 8-connected components
+ *   Sec. 3.4         island-parallel redraw with a ZipAR-style row window: step index
  *   Sec. 3.2 Step 1  y~ ~ M_q: the drafter's own sampling, on given logits
  *   Sec. 3.2 Step 7  y = D_r(x): stand-in, majority token of each r x r block
  *   Supp. "Sampling" temperature, top-k, classifier-free guidance of the sampler
@@ -55,7 +56,9 @@
  * and on hand-drawn shapes; the draft sampler against the pinned primitives
  * composed in the test and by chi-square over rounds; the down-sampler by
  * D_r(U_r(y)) = y, scipy.stats.mode on blocks without ties, and hand-written
- * blocks with ties.  The paper prints no worked numeric example for this
+ * blocks with ties; the island schedule by a time-stepped simulation of the
+ * rule, the closed form W + (H - 1) w of a full grid, and island size when the
+ * window spans the row.  The paper prints no worked numeric example for this
  * path, so no pin is a printed value.
  */
 #include <math.h>
@@ -366,6 +369,39 @@ int orc_islands(const uint8_t* in_rx, int H, int W, int32_t* labels, int32_t* ro
   }
   free(stack);
   return M;
+}
+
+/* Sec. 3.4, "within each island the ZipAR decoding strategy": the sequential
+ * target-model step at which each position of R_X is redrawn when the islands
+ * run concurrently and, inside an island, rows advance left to right with the
+ * row-window rule of ZipAR-w: a position may be decoded one step after its
+ * predecessor in the same row of the island, and one step after the row above
+ * (of the same island) has been decoded up to `window - 1` columns beyond it:
+ *   step(t) = 1 + max( step(previous position of the island in row i),
+ *                      max{ step(u) : u in the island, row(u) = i - 1,
+ *                                     col(u) <= col(t) + window - 1 } ),
+ * a maximum over nothing counting as 0.  (The paper names the strategy and the
+ * window, 16; this recurrence is the reading taken for it.)
+ *   labels [H*W] island numbers (0 outside R_X);  step [H*W] out, 0 outside R_X.
+ * Returns the number of sequential steps of the image, max step. */
+int orc_island_schedule(const int32_t* labels, int H, int W, int window, int32_t* step) {
+  int nfe = 0;
+  for (int i = 0; i < H; ++i)
+    for (int j = 0; j < W; ++j) {
+      const int m = labels[i * W + j];
+      step[i * W + j] = 0;
+      if (m <= 0) continue;
+      int before = 0;
+      for (int jj = 0; jj < j; ++jj) /* predecessor(s) in the same row */
+        if (labels[i * W + jj] == m && step[i * W + jj] > before) before = step[i * W + jj];
+      if (i > 0)
+        for (int jj = 0; jj < W && jj <= j + window - 1; ++jj)
+          if (labels[(i - 1) * W + jj] == m && step[(i - 1) * W + jj] > before)
+            before = step[(i - 1) * W + jj];
+      step[i * W + j] = before + 1;
+      if (before + 1 > nfe) nfe = before + 1;
+    }
+  return nfe;
 }
 
 /* ---------------------------------------------------------------- stages */
