@@ -465,6 +465,48 @@ def run_islands(args, cfg):
                          "unit": "GB/s", "frac": alg / (ms * 1e-3) / 1e9 / peak, "bytes_per_launch": alg,
                          "traffic": None},
             "cpu_baseline": cpu, "gpu_launches": ctx.kernel_launches() - launches0}), flush=True)
+        if B != cfg.B:
+            continue
+        # the schedule of the redraw: islands concurrently, a row window of 16 inside an island (ZipAR-16)
+        window = 16
+        step = torch.empty((B, cfg.H, cfg.W), dtype=torch.int32, device=dev)
+        n_steps = torch.empty((B,), dtype=torch.int32, device=dev)
+        e = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for s_ in range(W + K):
+            flush.zero_()
+            if s_ >= W:
+                e[s_ - W][0].record()
+            ctx.mulo_island_schedule(pb, labels, window, step, n_steps)
+            if s_ >= W:
+                e[s_ - W][1].record()
+        torch.cuda.synchronize()
+        ms = statistics.mean(a.elapsed_time(b) for a, b in e)
+        n_rx = int(out["n_expand"].sum().item())
+        acc = 1.0 - int(out["n_reject"].sum().item()) / positions
+        t_p, t_q = cfg.H * cfg.W, cfg.h * cfg.w
+        cpu = None
+        if not args.no_cpu_baseline:
+            lab = labels.cpu().numpy()
+            t0 = time.time()
+            total = sum(oracle.island_schedule(lab[b], window)[1] for b in range(B))
+            dt = time.time() - t0
+            assert total == int(n_steps.sum().item())
+            cpu = {"value": positions / dt, "unit": "positions/s", "cores": 1, "kind": "oracle",
+                   "sample": f"all {B} images", "seconds": dt}
+        alg = 2 * labels.numel() * 4 + n_steps.numel() * 4
+        print(json.dumps({
+            "stage": "mulo_island_schedule", "metric": "scheduled_positions_per_sec",
+            "value": positions / (ms * 1e-3), "unit": "positions/s", "ms_per_step": ms, "steps": K, "warmup": W,
+            "dtype": "int32", "data": "synthetic",
+            "config": {"workload": workload_desc(cfg), "images": B, "window": window,
+                       "positions_to_redraw_per_image": n_rx / B,
+                       "sequential_target_steps_per_image": int(n_steps.sum().item()) / B,
+                       "acceptance_rate": acc,
+                       "theoretical_speedup_S_T": t_p / ((1.0 - acc) * t_p + t_q)},
+            "roofline": {"bound": "hbm", "kernel": "k_island_schedule", "achieved": alg / (ms * 1e-3) / 1e9,
+                         "peak": peak, "unit": "GB/s", "frac": alg / (ms * 1e-3) / 1e9 / peak,
+                         "bytes_per_launch": alg, "traffic": None},
+            "cpu_baseline": cpu}), flush=True)
     ctx.close()
 
 

@@ -192,6 +192,21 @@ mulo_status mulo_local_reject_expand(mulo_ctx* ctx, const mulo_params* p,
                                      const uint32_t* reject_bits, const int32_t* first_reject,
                                      uint32_t* expand_bits, int32_t* n_expand, void* stream);
 
+/* Schedule of the redraw (Sec. 3.4): different islands are redrawn concurrently; within an
+ * island the target model advances row by row, left to right, with a ZipAR-style row window:
+ * a position may be decoded one step after the island's previous position in its row, and one
+ * step after the island's positions of the row above up to `window - 1` columns beyond it,
+ *   step(t) = 1 + max(step of the island's earlier positions in row i,
+ *                     step of the island's positions (i - 1, j') with j' <= j + window - 1).
+ * The paper names the strategy and the window (16); this recurrence is the reading taken.
+ * A full H x W island takes W + (H - 1) window steps instead of H W.  H * W <= 16384.
+ *   labels  [B, H, W]  in   island numbers from mulo_islands (0 outside R_X)
+ *   window             >= 1
+ *   step    [B, H, W]  out  1-based sequential target-model step of the position, 0 outside R_X
+ *   n_steps [B]        out  sequential steps the image needs (the largest step)               */
+mulo_status mulo_island_schedule(mulo_ctx* ctx, const mulo_params* p, const int32_t* labels,
+                                 int32_t window, int32_t* step, int32_t* n_steps, void* stream);
+
 /* Step 1 on given logits (Sec. 3.2): the drafter's own draw y~ ~ q, one token per low-res cell,
  * by inverse CDF in ascending token id over q = softmax(topk(l_q / T)) (same temperature and
  * top-k as the round).  The uniform is word 0 of the Philox stream with counter

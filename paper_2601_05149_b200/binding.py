@@ -24,7 +24,7 @@ EXPORTS = (
     "mulo_create", "mulo_destroy", "mulo_status_string", "mulo_workspace_bytes",
     "mulo_set_workspace", "mulo_poll_device_status", "mulo_poll_fallback_counts", "mulo_kernel_launches",
     "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only",
-    "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_islands", "mulo_sample_draft", "mulo_downsample", "mulo_resample",
+    "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_islands", "mulo_island_schedule", "mulo_sample_draft", "mulo_downsample", "mulo_resample",
     "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host", "mulo_round_static",
 )
 
@@ -218,6 +218,10 @@ class Context:
         _check(lib().mulo_local_reject_expand(self._ctx, C.byref(p), _dev(reject_bits),
                                               _dev(first_reject), _dev(expand_bits), _dev(n_expand),
                                               _stream(stream)), "mulo_local_reject_expand")
+
+    def mulo_island_schedule(self, p, labels, window, step, n_steps, stream=None):
+        _check(lib().mulo_island_schedule(self._ctx, C.byref(p), _dev(labels), C.c_int32(int(window)), _dev(step),
+                                          _dev(n_steps), _stream(stream)), "mulo_island_schedule")
 
     def mulo_sample_draft(self, p, draft_logits_lo, draft_tok_lo, stream=None):
         _check(lib().mulo_sample_draft(self._ctx, C.byref(p), _dev(draft_logits_lo), _dev(draft_tok_lo),

@@ -782,6 +782,27 @@ mulo_status mulo_upsample_pool(mulo_ctx* ctx, const mulo_params* p, const void* 
   return launched(ctx, 1);
 }
 
+mulo_status mulo_island_schedule(mulo_ctx* ctx, const mulo_params* p, const int32_t* labels, int32_t window,
+                                 int32_t* step, int32_t* n_steps, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!labels || !step || !n_steps || window < 1) return MULO_ERR_INVALID_ARG;
+  if ((size_t)p->H * p->W > (size_t)kIslandMaxCells) return MULO_ERR_UNSUPPORTED;
+  if (p->B == 0) return MULO_OK;
+  ScheduleArgs a;
+  a.H = p->H; a.W = p->W; a.window = window > p->W ? p->W : window;
+  a.labels = labels; a.step = step; a.n_steps = n_steps;
+  const size_t smem = (size_t)4 * p->W * sizeof(int);
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(k_island_schedule, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return MULO_ERR_CUDA;
+  }
+  k_island_schedule<<<p->B, kScheduleThreads, smem, (cudaStream_t)stream>>>(a);
+  return launched(ctx, 1);
+}
+
 mulo_status mulo_sample_draft(mulo_ctx* ctx, const mulo_params* p, const void* draft_logits_lo,
                               int32_t* draft_tok_lo, void* stream) {
   if (!ctx) return MULO_ERR_INVALID_ARG;

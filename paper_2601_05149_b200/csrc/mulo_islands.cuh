@@ -205,4 +205,73 @@ __global__ void __launch_bounds__(kIslandThreads) k_islands(IslandArgs a) {
   }
 }
 
+// Island schedule (Sec. 3.4: islands redrawn concurrently, a ZipAR-style row window inside an island):
+// the sequential step at which each position of R_X is decoded,
+//   step(t) = 1 + max(step of the island's earlier positions in the row,
+//                     step of the island's positions in the row above up to column col(t) + window - 1).
+// Along a row the recurrence s_k = max(s_{k-1} + 1, d_k) has the closed form
+// s_k = max_{l <= k} (d_l + k - l), so the positions of a row are independent of one another: one CTA per
+// image, one thread per column, the rows in sequence.
+struct ScheduleArgs {
+  int H, W, window;
+  const int32_t* labels;   // [B, H, W]
+  int32_t* step;           // [B, H, W]
+  int32_t* n_steps;        // [B]
+};
+
+constexpr int kScheduleThreads = 256;
+
+__global__ void __launch_bounds__(kScheduleThreads) k_island_schedule(ScheduleArgs a) {
+  extern __shared__ int sched_smem[];
+  const int H = a.H, W = a.W, b = blockIdx.x, tid = threadIdx.x;
+  int* const lab_up = sched_smem;           // labels of row i - 1
+  int* const step_up = sched_smem + W;      // steps of row i - 1
+  int* const lab = sched_smem + 2 * W;      // labels of row i
+  int* const dep = sched_smem + 3 * W;      // d_k of row i: 1 + what the row above demands
+  __shared__ int s_max;
+  if (tid == 0) s_max = 0;
+  const int32_t* labels = a.labels + (size_t)b * H * W;
+  int32_t* step = a.step + (size_t)b * H * W;
+  int local_max = 0;
+  for (int i = 0; i < H; ++i) {
+    __syncthreads();   // the previous row's results are in step_up / lab_up
+    for (int j = tid; j < W; j += kScheduleThreads) lab[j] = labels[(size_t)i * W + j];
+    __syncthreads();
+    for (int j = tid; j < W; j += kScheduleThreads) {
+      const int m = lab[j];
+      int d = 1;
+      if (m > 0 && i > 0) {
+        // steps grow along a row of an island: its last position at or before column j + window - 1
+        for (int jj = min(W - 1, j + a.window - 1); jj >= 0; --jj)
+          if (lab_up[jj] == m) {
+            d = step_up[jj] + 1;
+            break;
+          }
+      }
+      dep[j] = d;
+    }
+    __syncthreads();
+    for (int j = tid; j < W; j += kScheduleThreads) {
+      const int m = lab[j];
+      int s = 0;
+      if (m > 0) {
+        int behind = 0;   // k - l: positions of the island between column jj and column j
+        for (int jj = j; jj >= 0; --jj)
+          if (lab[jj] == m) {
+            s = max(s, dep[jj] + behind);
+            ++behind;
+          }
+      }
+      step[(size_t)i * W + j] = s;
+      local_max = max(local_max, s);
+      // becomes the row above (nobody reads step_up / lab_up any more in this row)
+      step_up[j] = s;
+      lab_up[j] = m;
+    }
+  }
+  atomicMax(&s_max, local_max);
+  __syncthreads();
+  if (tid == 0) a.n_steps[b] = s_max;
+}
+
 }  // namespace mulo

@@ -103,6 +103,53 @@ def test_islands_of_a_real_round(ctx):
     check_against_oracle(ctx, mask, max_islands=256)
 
 
+def schedule_both(ctx, mask, window):
+    B, H, W = mask.shape
+    p = binding.make_params(B, H, W, 8, 1, binding.F32)
+    labels, _, _, _ = run_islands(ctx, mask, 0)
+    step = torch.full((B, H, W), -7, dtype=torch.int32, device="cuda")
+    n = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    ctx.mulo_island_schedule(p, torch.from_numpy(labels).cuda(), window, step, n)
+    torch.cuda.synchronize()
+    step, n = step.cpu().numpy(), n.cpu().numpy()
+    for b in range(B):
+        want, nfe = oracle.island_schedule(oracle.islands(mask[b])[0], window)
+        np.testing.assert_array_equal(step[b], want)
+        assert n[b] == nfe
+    return step, n
+
+
+@pytest.mark.parametrize("shape", [(2, 1, 1), (2, 1, 40), (2, 9, 1), (3, 17, 33), (4, 64, 64), (2, 40, 70),
+                                   (1, 16, 1024), (1, 128, 128)])
+@pytest.mark.parametrize("window", [1, 3, 16])
+def test_schedule_random_masks(ctx, shape, window):
+    rng = np.random.default_rng(shape[1] * 77 + shape[2] + window)
+    for density in (0.1, 0.5, 0.9):
+        mask = (rng.random(shape) < density).astype(np.uint8)
+        schedule_both(ctx, mask, window)
+
+
+def test_schedule_closed_forms(ctx):
+    H, W = 32, 48
+    mask = np.zeros((3, H, W), np.uint8)
+    mask[0] = 1                      # one island covering the grid
+    mask[1, 4:12, 10:30] = 1         # a solid block
+    step, n = schedule_both(ctx, mask, 16)
+    assert list(n) == [W + (H - 1) * 16, 20 + 7 * 16, 0]
+    step, n = schedule_both(ctx, mask, 1000)          # window beyond the row: raster order inside an island
+    assert list(n) == [H * W, 8 * 20, 0]
+
+
+def test_schedule_of_a_real_round(ctx):
+    cfg = synth.RoundConfig("sched", B=4, H=32, W=32, V=512, dtype="bf16", top_k=64, sigma=0.3, radius=1,
+                            seed=4343)
+    batch = pu.build_batch(cfg)
+    g = pu.gpu_round(ctx, cfg, batch)
+    mask = g["expand"].astype(np.uint8)
+    step, n = schedule_both(ctx, mask, 16)
+    assert (n <= mask.reshape(cfg.B, -1).sum(1)).all() and (n > 0).any()
+
+
 def test_limits_are_refused_before_launch(ctx):
     p = binding.make_params(1, 129, 128, 8, 1, binding.F32)
     bits = torch.zeros((1, 129, 4), dtype=torch.int32, device="cuda")
