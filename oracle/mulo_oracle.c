@@ -79,7 +79,7 @@
 
 /* borderline flags reported per position */
 #define ORC_FLAG_ACCEPT_EDGE 1u /* |u - thr| < 1e-6 (or pooled mass within 1e-6 rel. of tau) */
-#define ORC_FLAG_CDF_EDGE 2u    /* u' within 1e-6 of an edge of the chosen CDF bin   */
+#define ORC_FLAG_CDF_EDGE 2u    /* u' Z_w within 1e-6 (of mass) of an edge of the chosen CDF bin */
 #define ORC_FLAG_POOL_EDGE 4u   /* some prefix mass c_j within 1e-6 of delta          */
 
 typedef struct {
@@ -491,7 +491,11 @@ static void visit_position(const orc_params* P, const float* zt, const double* q
     t1 = orc_inverse_cdf(wts, V, u[1], &Zw, &eg);
   }
   out->tok_residual = t1;
-  out->flag_residual = eg < 1e-6 ? ORC_FLAG_CDF_EDGE : 0u;
+  /* The edge test of a draw is taken in units of probability mass, |u Z_w - C(x)| < 1e-6:
+   * the probabilities are only defined to the stated relative tolerance, so a
+   * residual that holds less than 1e-6 of mass decides nothing and is always
+   * borderline.  (Z_w = 1 for the target weights: there both readings agree.) */
+  out->flag_residual = eg * Zw < 1e-6 ? ORC_FLAG_CDF_EDGE : 0u;
   orc_residual_weights(p_prime, q, V, 0.0, wts);
   int t0 = orc_inverse_cdf(wts, V, u[2], &Zw, &eg);
   out->tok_target = t0;

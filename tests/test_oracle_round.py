@@ -31,6 +31,29 @@ def _image(cfg, b=0):
 SMALL = synth.RoundConfig("small", B=1, H=8, W=8, V=256, dtype="f32", sigma=0.7, radius=1, seed=11)
 
 
+def test_a_residual_with_next_to_no_mass_is_flagged_borderline(orc):
+    """Target one ulp away from the draft in a single logit: the residual max(0, p - q) holds about 1e-8 of
+    mass, so its normalised CDF means nothing at the tolerance of the probabilities -- every residual draw
+    there carries the CDF-edge flag.  With the target equal to the draft the residual is exactly empty, the
+    draw falls back to the target weights (mass 1) and is flagged only by the usual edge test."""
+    cfg = dataclasses.replace(SMALL, dtype="f32", sigma=0.0, resample_mode=orc.RESAMPLE_RESIDUAL_ALL, radius=8,
+                              clip_before_first=0)
+    cond, uncond, draft, tok = _image(cfg)
+    cond = cond.copy()
+    cond[:, :, 5] = np.nextafter(cond[:, :, 5], np.float32(np.inf))
+    # force one rejection so that R_X (radius 8, no clipping) covers the grid
+    cond[0, 0, :] = -30.0
+    cond[0, 0, (int(tok[0, 0]) + 1) % cfg.V] = 30.0
+    out = orc.round_image(_params(orc, cfg), cond, None, draft, tok)
+    assert out["reject"][0, 0] == 1 and out["expand"].all()
+    near = np.ones((cfg.H, cfg.W), bool)
+    near[0, 0] = False
+    assert (out["flags"][near] & orc.FLAG_CDF_EDGE).all()
+    assert not (out["flags"][0, 0] & orc.FLAG_CDF_EDGE)          # a residual with all the mass: decided
+    same = orc.round_image(_params(orc, cfg), np.kron(draft, np.ones((2, 2, 1), np.float32)), None, draft, tok)
+    assert same["reject"].sum() == 0
+
+
 @pytest.mark.parametrize("dtype,top_k", [("f32", 0), ("bf16", 0), ("bf16", 40)])
 def test_target_equal_to_draft_accepts_everything(orc, dtype, top_k):
     cfg = dataclasses.replace(SMALL, dtype=dtype, top_k=top_k, sigma=0.0)
