@@ -335,3 +335,30 @@ def test_fast_path_adapts_to_rows_that_are_not_normal(ctx):
     assert lost < 0.6 * rows, (lost, rows)      # every CTA loses its first few parents while it adapts
     o = pu.oracle_images(cfg, batch, [0, cfg.B - 1])
     pu.check_round(cfg, g, o)
+
+
+@pytest.mark.parametrize("fast", [True, False])
+def test_residual_for_all_with_near_one_hot_rows(ctx, fast):
+    """Cubed logits make target and draft near one-hot; drawing EVERY position of R_X from the residual then
+    asks, at accepted positions, for a draw from max(0, p - q) with next to no mass.  In fp32 that residual is
+    empty (the draw falls back to the target weights), in fp64 it is rounding dust: the oracle flags such
+    draws (edge test in units of probability mass), and the outputs may differ only there.  No budget on how
+    many: the case is ill-posed by construction."""
+    cfg = synth.RoundConfig("onehot", B=2, H=8, W=24, V=4096, r=2, dtype="bf16", top_k=64, cfg_scale=7.5,
+                            sigma=2.0, radius=2, resample_mode=binding.RESAMPLE_RESIDUAL_ALL, seed=219012)
+    batch = pu.build_batch(cfg)
+    for k in ("cond", "uncond", "draft_lo"):
+        batch[k] = (batch[k].float() ** 3).to(batch[k].dtype).contiguous()
+    batch["tok_lo"] = batch["draft_lo"].float().argmax(-1).to(torch.int32).contiguous()
+    ctx.set_general_path_only(not fast)
+    try:
+        g = pu.gpu_round(ctx, cfg, batch)
+    finally:
+        ctx.set_general_path_only(False)
+    o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
+    differ = flagged = 0
+    for b in range(cfg.B):
+        e, f = pu.compare_image(cfg, g, b, o[b], 2e-3)     # raises where an unflagged position differs
+        differ += e
+        flagged += f
+    assert flagged > 0
