@@ -224,7 +224,9 @@ __global__ void __launch_bounds__(kThreads) k_verify_rows(RowKernelArgs a) {
 __global__ void __launch_bounds__(kThreads) k_verify_failed(RowKernelArgs a, const int32_t* fail_list,
                                                             const uint32_t* fail_count) {
   __shared__ BlockScratch bs;
+  extern __shared__ __align__(16) unsigned char dyn[];
   const DevParams& P = a.P;
+  PoolSmem ps = carve_pool(P, dyn);
   const int N = P.H * P.W;
   const size_t total = (size_t)P.B * N;
   const size_t n = min((size_t)*fail_count, total);
@@ -244,9 +246,8 @@ __global__ void __launch_bounds__(kThreads) k_verify_failed(RowKernelArgs a, con
     RowSrc tr = target_row(a, g);
     PositionOut o;
     const int mode = P.resample_mode;
-    PoolSmem none = {nullptr, nullptr};
-    dense_position(P, tr, qr, sq, tok, nullptr, (uint32_t)b + P.image_offset, (uint32_t)t, true, 0,
-                   [mode](int acc) { return draws_for(mode, acc); }, bs, none, a.dev_status, o);
+    dense_position(P, tr, qr, sq, tok, a.nn, (uint32_t)b + P.image_offset, (uint32_t)t, true, 0,
+                   [mode](int acc) { return draws_for(mode, acc); }, bs, ps, a.dev_status, o);
     if (threadIdx.x == 0) {
       a.flags[g] = o.accepted ? 0 : 1;
       a.cand_res[g] = o.tok_residual;
@@ -695,7 +696,9 @@ static double inv_norm_cdf(double p) {
 // Fills `s` and returns the dynamic shared memory the streaming kernel needs, or 0 if these
 // parameters are not eligible (then the general kernel runs).
 static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s) {
-  if (d.top_k <= 0 || d.pool_k > 1) return 0;
+  if (d.top_k <= 0) return 0;
+  // pooling keeps a bitmap of the pooled token ids in the row's selection scratch (2 KB)
+  if (d.pool_k > 1 && d.V > 16384) return 0;
   const int V = d.V, k = d.top_k;
   if (V < 1024 || 1 + d.r * d.r > kMaxRowsPerParent) return 0;
   // candidates aimed for beyond k: about six standard deviations of the count of entries
@@ -730,9 +733,9 @@ static size_t plan_stream(const mulo_ctx* ctx, const DevParams& d, StreamArgs* s
   return dyn;
 }
 
-template <bool BF16, bool HAS_U, bool SAMPLE = false>
+template <bool BF16, bool HAS_U, bool SAMPLE = false, bool POOL = false>
 static bool launch_stream_t(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn, cudaStream_t st) {
-  auto kern = k_round_stream<BF16, HAS_U, SAMPLE>;
+  auto kern = k_round_stream<BF16, HAS_U, SAMPLE, POOL>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
     cudaGetLastError();
     return false;
@@ -750,6 +753,13 @@ static bool launch_stream_t(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn
 
 static bool launch_stream(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn, cudaStream_t st) {
   const bool hu = s.uncond != nullptr;
+  if (s.P.pool_k > 1) {
+    if (s.P.bf16)
+      return hu ? launch_stream_t<true, true, false, true>(ctx, s, dyn, st)
+                : launch_stream_t<true, false, false, true>(ctx, s, dyn, st);
+    return hu ? launch_stream_t<false, true, false, true>(ctx, s, dyn, st)
+              : launch_stream_t<false, false, false, true>(ctx, s, dyn, st);
+  }
   if (s.P.bf16) return hu ? launch_stream_t<true, true>(ctx, s, dyn, st) : launch_stream_t<true, false>(ctx, s, dyn, st);
   return hu ? launch_stream_t<false, true>(ctx, s, dyn, st) : launch_stream_t<false, false>(ctx, s, dyn, st);
 }
@@ -1000,6 +1010,7 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   a.dev_status = w.status;
   const size_t dyn = pool_smem_bytes(a.P);
   if (!raise_smem(k_verify_rows<true>, dyn, ctx)) return MULO_ERR_UNSUPPORTED;
+  if (!raise_smem(k_verify_failed, dyn, ctx)) return MULO_ERR_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
   const bool timed = ctx->ev_used + 2 <= ctx->ev.size();
   if (timed) cudaEventRecord(ctx->ev[ctx->ev_used], st);
@@ -1010,6 +1021,7 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   if (sdyn) {
     sa.P = a.P;
     sa.cond = a.cond; sa.uncond = a.uncond; sa.draft = a.draft; sa.draft_tok_lo = draft_tok_lo;
+    sa.nn = a.nn;
     sa.p_tok = p_tok; sa.q_tok = q_tok; sa.accept_prob = accept_prob;
     sa.flags = w.flags; sa.cand_res = w.cand_res; sa.cand_tgt = w.cand_tgt;
     sa.dev_status = w.status;
@@ -1018,7 +1030,7 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
     if (cudaMemsetAsync(w.status + kFailCount, 0, sizeof(uint32_t), st) != cudaSuccess) return MULO_ERR_CUDA;
     fast = launch_stream(ctx, sa, sdyn, st);
     // the rows the streaming kernel gave up on (usually a handful, often none)
-    if (fast) k_verify_failed<<<2 * ctx->sm_count, kThreads, 0, st>>>(a, w.fail_list, w.status + kFailCount);
+    if (fast) k_verify_failed<<<2 * ctx->sm_count, kThreads, dyn, st>>>(a, w.fail_list, w.status + kFailCount);
   }
   if (!fast) k_verify_rows<true><<<p->B * a.P.h * a.P.w, kThreads, dyn, st>>>(a);
   if (timed) {

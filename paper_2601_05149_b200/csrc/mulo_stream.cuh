@@ -133,6 +133,7 @@ struct StreamArgs {
   const char* uncond;
   const char* draft;
   const int32_t* draft_tok_lo;
+  const uint16_t* nn;    // pooling: [V, pool_k] neighbour lists (entry 0 of a row is the token itself)
   int32_t* sample_out;   // sampling mode: [B, h, w] the drafter's own draw per low-res cell
   float* p_tok;
   float* q_tok;
@@ -225,6 +226,11 @@ struct StreamSmem {
   Predictor pred[2];   // 0: draft rows, 1: target rows
   float red[kSWarps][2];   // bootstrap statistics
   double e_tok;        // exp(z_tok - m_p) of the current target row
+  // pooling (Eq. 3-4): warp totals of the prefix scan, first list index whose prefix mass reaches
+  // delta, the pooled mass c_J
+  double wsum[kSWarps];
+  double cJ;
+  int first_bad;
   // the current parent
   double Zq, q_tok;
   float theta_q, m_q, invZq;
@@ -442,9 +448,13 @@ struct Sel {
 // SAMPLE = true turns the kernel into the drafter's own sampling (Sec. 3.2 Step 1): only the draft
 // rows are streamed (one row per "parent"), and instead of verifying children one warp draws
 // y~ ~ q from the row's candidate list with word 0 of the tag-1 Philox stream.
-template <bool BF16, bool HAS_U, bool SAMPLE = false>
+// POOL = true adds the probability pooling of Eq. 3-4 to a target row: the pooled mass of the
+// codebook neighbours of x~ enters the acceptance test, and the redraw uses p' (neighbours' mass
+// moved onto x~).
+template <bool BF16, bool HAS_U, bool SAMPLE = false, bool POOL = false>
 __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_constant__ StreamArgs a) {
   static_assert(!(SAMPLE && HAS_U), "draft rows have no unconditional stream");
+  static_assert(!(SAMPLE && POOL), "the drafter's own draw has no pooling");
   constexpr int EPL = BF16 ? 8 : 4;        // entries per lane visit (16 bytes of the conditional row)
   constexpr int PIECE = 32 * EPL;          // entries per 32-lane piece
   constexpr int SEG = kPPW * PIECE;        // entries of the row that one segment covers
@@ -652,6 +662,12 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
 #pragma unroll
           for (int j = 0; j < EPL; ++j)
             if (z[i][j] >= pivot) mask[i] |= 1u << j;
+          // pooling moves mass onto x~, so x~ gets an entry whatever its value (one that is below
+          // the pivot counts for nothing until then: no histogram bin, e = 0)
+          if (POOL && !IS_Q) {
+            const unsigned d = (unsigned)(sm.tok - (c * a.chunk + e));
+            if (d < (unsigned)EPL) mask[i] |= 1u << d;
+          }
         }
       }
       // one warp scan for both pieces' counts (16 bits each); lane 31 then claims one run of the
@@ -710,7 +726,14 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     auto tally = [&](float zz) {
       mx = fmaxf(mx, zz);
       const float fb = __fmul_rn(__fsub_rn(zz, pivot), inv_w);
-      if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+      if (POOL && !IS_Q) {   // the list may hold x~ from below the pivot: not a candidate
+        if (zz >= pivot) {
+          ++mine;
+          if (fb < (float)kHistBins) atomicAdd(&rs.hist[(int)fb], 1u);
+        }
+      } else if (fb < (float)kHistBins) {
+        atomicAdd(&rs.hist[(int)fb], 1u);
+      }
     };
     auto tally_pair = [&](int first, int sl, int cn) {
       float z0, z1;
@@ -727,7 +750,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     for (int c = grp; c < a.n_chunks; c += groups) {
       const ushort2 r = run[c * kSWarps + warp];
       const int cn = r.y;
-      if (sub == 0) mine += (unsigned)cn;
+      if (!(POOL && !IS_Q) && sub == 0) mine += (unsigned)cn;
       for (int sl = 2 * sub; sl < cn; sl += 4 * seg_lanes) {
         tally_pair(r.x, sl, cn);
         if (sl + 2 * seg_lanes < cn) tally_pair(r.x, sl + 2 * seg_lanes, cn);
@@ -811,7 +834,8 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     // e of one entry (value z at index `at`); the crossing bin's entries are set aside
     auto one = [&](int seg, int at, float z, float& acc) -> float {
       const float fb = __fmul_rn(__fsub_rn(z, pivot), inv_w);
-      const int bin = fb < (float)kHistBins ? (int)fb : kHistBins;
+      int bin = fb < (float)kHistBins ? (int)fb : kHistBins;
+      if (POOL && !IS_Q && z < pivot) bin = -1;   // x~ from below the pivot: e = 0
       float e = 0.f;
       if (bin >= s.bstar) e = fast_exp(z, s.m);
       if (bin == s.bstar) {
@@ -991,6 +1015,81 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     pp.z_tok = load1(tr, sm.tok);
   };
 
+  // Eq. 3-4 for the target row at position g, after its theta, m and Z_p are known (all threads;
+  // four block barriers).  c_j = sum_{i<=j} p(n_i) along the neighbour list of x~; the leading
+  // run with c_j < delta is pooled: J entries, mass c_J.  Leaves a bitmap of the pooled token ids
+  // in the (by now unused) selection scratch of the row.
+  auto pool_phase = [&](float theta, float m, double Zp, size_t g, double& cJ, int& J) {
+    const int nb = P.pool_k - 1;
+    const uint16_t* row = a.nn + (size_t)sm.tok * P.pool_k;
+    uint32_t* const bitmap = reinterpret_cast<uint32_t*>(&rs);
+    static_assert(sizeof(RowState::hist) + sizeof(RowState::member_z) + sizeof(RowState::member_at) +
+                      sizeof(RowState::member_seg) >= 16384 / 8,
+                  "the bitmap of a 16384-entry vocabulary must fit the selection scratch");
+    const RowSrc tr = {a.cond + g * (size_t)P.V * esz, HAS_U ? a.uncond + g * (size_t)P.V * esz : nullptr,
+                       P.cfg_scale, P.invT, P.V, BF16};
+    __syncthreads();   // every warp is done with the set-aside entries
+    for (int x = tid; x < (P.V + 31) / 32; x += kSThreads) bitmap[x] = 0u;
+    if (tid == 0) {
+      sm.first_bad = nb;
+      sm.cJ = 0.0;
+    }
+    constexpr int PER = 8;   // list entries per thread: pool_k <= 2048
+    const int per = (nb + kSThreads - 1) / kSThreads;
+    const int j0 = tid * per;
+    double loc[PER];
+    int ids[PER];
+    double run = 0.0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      ids[i] = -1;
+      loc[i] = run;
+      if (i < per && j0 + i < nb) {
+        int id = row[j0 + i + 1];
+        if (id >= P.V) {
+          atomicOr(a.dev_status, MULO_DEV_BAD_TOKEN);
+          id = P.V - 1;
+        }
+        ids[i] = id;
+        const float z = load1(tr, id);
+        run += (z >= theta) ? (double)expf(__fsub_rn(z, m)) / Zp : 0.0;
+        loc[i] = run;
+      }
+    }
+    double inc = run;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double v = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += v;
+    }
+    if (lane == 31) sm.wsum[warp] = inc;
+    // mass before this thread's entries: the lanes below (taken from the scan, not as inc - run: a
+    // large entry in `run` would cancel the small masses before it), then the warps below
+    double carry = __shfl_up_sync(kFull, inc, 1);
+    if (lane == 0) carry = 0.0;
+    __syncthreads();
+    {
+      double below = 0.0;
+      for (int w = 0; w < warp; ++w) below += sm.wsum[w];
+      carry = below + carry;
+    }
+    int bad = nb;
+#pragma unroll
+    for (int i = PER - 1; i >= 0; --i)
+      if (ids[i] >= 0 && !(carry + loc[i] < P.pool_delta)) bad = j0 + i;
+    if (bad < nb) atomicMin(&sm.first_bad, bad);
+    __syncthreads();
+    J = sm.first_bad;
+#pragma unroll
+    for (int i = 0; i < PER; ++i)
+      if (ids[i] >= 0 && j0 + i < J) {
+        atomicOr(&bitmap[ids[i] >> 5], 1u << (ids[i] & 31));
+        if (j0 + i == J - 1) sm.cJ = carry + loc[i];
+      }
+    __syncthreads();
+    cJ = sm.cJ;
+  };
+
   // One thread, a phase ahead of prepare_row: asks L2 for the lines that hold the logit of x~ at
   // the next target position, so that the load there does not wait on HBM.
   auto prefetch_row = [&](int child) {
@@ -1133,14 +1232,28 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
         const bool ok_sel = ok;   // the predictor learns from it while the draws run
         const int t = (sm.ca * P.r + child / P.r) * P.W + sm.cc * P.r + child % P.r;
         const size_t g = (size_t)sm.b * P.H * P.W + t;
+        double cJ = 0.0;   // pooled mass of the neighbours of x~ (Eq. 3-4), J of them
+        int J = 0;
+        if constexpr (POOL) {
+          if (ok) {   // block-uniform
+            pool_phase(theta, s.m, Zp, g, cJ, J);
+          }
+        }
+        const bool pooled = POOL && ok && J > 0;
         int draws = 0;
         float invZp = 0.f, invZq = 0.f;
+        double mass = 0.0;   // P of Eq. 3: own probability plus pooled mass
         if (ok) {
           // ---- the decision (Eq. 1 / Eq. 5), the same in every warp
           const double e_tok = (pp.z_tok >= theta) ? sm.e_tok : 0.0;
           const double q_tok = sm.q_tok;
           int accepted;
-          if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = e_tok >= P.tau * Zp;
+          if (pooled) {
+            mass = e_tok / Zp + cJ;
+            if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = mass >= P.tau;
+            else if (q_tok <= 0.0) accepted = mass > 0.0;
+            else accepted = uniform24(pp.rnd[0]) < fmin(1.0, mass / q_tok);
+          } else if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = e_tok >= P.tau * Zp;
           else if (q_tok <= 0.0) accepted = e_tok > 0.0;
           else accepted = uniform24(pp.rnd[0]) * q_tok * Zp < e_tok;
           draws = draws_for(P.resample_mode, accepted);
@@ -1151,7 +1264,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
             if (a.p_tok) a.p_tok[g] = (float)(e_tok / Zp);
             if (a.q_tok) a.q_tok[g] = (float)q_tok;
             if (a.accept_prob) {
-              const double p = e_tok / Zp;
+              const double p = pooled ? mass : e_tok / Zp;
               double thr;
               if (P.accept_mode == MULO_ACCEPT_THRESHOLD) thr = p;
               else if (q_tok <= 0.0) thr = p > 0.0 ? 1.0 : 0.0;
@@ -1186,7 +1299,39 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
           return w;
         };
         auto w_target = [&](int i) { return __uint_as_float(cand[i].x); };
-        if (draws & kDrawResidual) {   // block-uniform
+        if (pooled) {   // block-uniform
+          // p' in place: the pooled neighbours lose their mass, x~ gets P; the per-segment sums of
+          // p' (target draw, and the fallback of a residual without mass) and of the residual
+          const uint32_t* const bitmap = reinterpret_cast<const uint32_t*>(&rs);
+          const unsigned e_pool = __float_as_uint((float)(mass * Zp));
+          const int tok = sm.tok;
+          for (int c0 = 0; c0 < a.n_chunks; c0 += groups) {
+            const int c = c0 + grp;
+            const bool has = c < a.n_chunks;
+            const int seg = c * kSWarps + warp;
+            float acc_b = 0.f, acc_c = 0.f;
+            if (has) {
+              const ushort2 r = tseg[seg];
+              const int qfirst = qseg[seg].x;
+              for (int sl = sub; sl < (int)r.y; sl += seg_lanes) {
+                uint2 en = cand[r.x + sl];
+                const int id = (int)en.y;
+                if (id == tok) en.x = e_pool;
+                else if ((bitmap[id >> 5] >> (id & 31)) & 1u) en.x = 0u;
+                cand[r.x + sl].x = en.x;
+                acc_c += __uint_as_float(en.x);
+                if (draws & kDrawResidual) acc_b += w_entry(en.x, en.y, qfirst);
+              }
+            }
+            __syncwarp();
+            acc_b = seg_lanes_sum(acc_b, seg_lanes);
+            acc_c = seg_lanes_sum(acc_c, seg_lanes);
+            if (sub == 0 && has) {
+              seg_b[seg] = acc_b;
+              seg_c[seg] = acc_c;
+            }
+          }
+        } else if (draws & kDrawResidual) {   // block-uniform
           for (int c0 = 0; c0 < a.n_chunks; c0 += groups) {
             const int c = c0 + grp;
             const bool has = c < a.n_chunks;

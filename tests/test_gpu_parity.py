@@ -91,19 +91,27 @@ def test_identity_target_equals_draft(ctx):
 
 def test_stages_equal_fused(ctx):
     """upsample_pool -> verify -> local_reject_expand -> resample gives exactly
-    the fused round; each stage is also checked against the oracle."""
+    the fused round of the general path; each stage is also checked against the oracle."""
     import oracle as orc
     for cfg in (dataclasses.replace(TINY, dtype="bf16", top_k=40, cfg_scale=3.0, radius=2, seed=150),
                 dataclasses.replace(TINY, V=2048, top_k=300, pool_k=128, dtype="bf16", seed=151,
                                     resample_mode=binding.RESAMPLE_ISOLATED_RESIDUAL)):
         batch = pu.build_batch(cfg)
-        f = pu.gpu_round(ctx, cfg, batch)
+        # the stages run the general routines: bit for bit the fused round on the general path ...
+        ctx.set_general_path_only(True)
+        try:
+            f = pu.gpu_round(ctx, cfg, batch)
+        finally:
+            ctx.set_general_path_only(False)
         s = pu.gpu_stages(ctx, cfg, batch)
         for k in ("out_tok", "reject_bits", "expand_bits", "n_reject", "n_expand", "first_reject",
                   "p_tok", "q_tok", "accept_prob"):
             assert np.array_equal(f[k], s[k]), k
         o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
         pu.check_round(cfg, s, o)
+        # ... and the fused round as it runs by default (the streaming kernel where it applies) meets
+        # the same bar against the oracle
+        pu.check_round(cfg, pu.gpu_round(ctx, cfg, batch), o)
         for b in range(cfg.B):
             up = orc.upsample_pool_image(pu.orc_params(cfg, b), synth.to_numpy_logits(batch["draft_lo"][b]),
                                          batch["tok_lo"][b].cpu().numpy())
@@ -362,3 +370,27 @@ def test_residual_for_all_with_near_one_hot_rows(ctx, fast):
         differ += e
         flagged += f
     assert flagged > 0
+
+
+@pytest.mark.parametrize("scale,pool_k,delta", [(4.0, 2048, 0.01), (1.0, 1000, 0.1), (0.2, 500, 0.3)])
+def test_pooling_on_the_streaming_path(ctx, scale, pool_k, delta):
+    """Eq. 3-4 inside the streaming kernel (top-k on, V <= 16384).  With logits scaled up the row is peaked:
+    the pooled prefix then adds masses of 1e-19 before an entry of 0.7, which the prefix sums must keep."""
+    cfg = synth.RoundConfig("poolfast", B=2, H=8, W=12, V=4096, r=2, dtype="bf16", top_k=1024, cfg_scale=7.5,
+                            sigma=1.0, radius=1, clip_before_first=0, pool_k=pool_k, pool_delta=delta,
+                            resample_mode=binding.RESAMPLE_ISOLATED_RESIDUAL, seed=305057)
+    batch = pu.build_batch(cfg)
+    for k in ("cond", "uncond", "draft_lo"):
+        batch[k] = (batch[k].float() * scale).to(batch[k].dtype).contiguous()
+    p = binding.params_from_config(cfg)
+    ctx.ensure_workspace(p)
+    ctx.mulo_sample_draft(p, batch["draft_lo"], batch["tok_lo"])     # draft tokens with q > 0 under the new logits
+    torch.cuda.synchronize()
+    n0 = ctx.kernel_launches()
+    g = pu.gpu_round(ctx, cfg, batch)
+    assert ctx.kernel_launches() - n0 == 3                            # streaming kernel, its list, the mask kernel
+    o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
+    pu.check_round(cfg, g, o)
+    pooled = sum(int((o[b]["accept_prob"] > o[b]["p_tok"] / np.maximum(o[b]["q_tok"], 1e-300) * (1 + 1e-9)).sum())
+                 for b in range(cfg.B))
+    assert pooled > 0                                                 # some position did gain pooled mass
