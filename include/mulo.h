@@ -133,11 +133,11 @@ mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags
 mulo_status mulo_poll_fallback_counts(mulo_ctx* ctx, void* stream, uint32_t counts[5]);
 /* Number of kernels this context has launched so far. */
 mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
-/* mulo_round picks between two row kernels: a fast one for rows with top-k on and pooling
- * off (each row streamed once, work done on the few thousand entries near and above the
- * top-k threshold; a row it cannot handle is redone by the general routines) and the general
- * one.  Both compute the same function.  `on` != 0 makes this context always use the general
- * kernel (for testing and comparison). */
+/* mulo_round and mulo_sample_draft pick between two row kernels: a fast one for rows with
+ * top-k on (V >= 1024; with pooling, V <= 16384; each row streamed once, work done on the few
+ * thousand entries near and above the top-k threshold; a row it cannot handle is redone by
+ * the general routines) and the general one.  Both compute the same function.  `on` != 0
+ * makes this context always use the general kernel (for testing and comparison). */
 mulo_status mulo_set_general_path_only(mulo_ctx* ctx, int on);
 /* Optional device timing of the fused row kernel (the launch that reads the logits):
  * mulo_set_timing prepares CUDA event pairs for up to max_launches (<= 4096) calls of
