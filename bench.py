@@ -586,6 +586,50 @@ def run_draft_io(args, cfg):
     ctx.close()
 
 
+def run_driver(args, cfg):
+    """The host loop over rounds (draft draw, fused round, islands, redraw schedule, down-sampled prefix) on
+    fresh synthetic logits per round: one JSON line per round with what the paper's latency analysis uses,
+    then one line with the device time of the library's own launches per round.  Single GPU."""
+    from paper_2601_05149_b200 import binding, driver
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the driver has no CPU path")
+    torch.cuda.set_device(0)
+    ctx = binding.Context(0)
+    d = driver.RoundDriver(cfg, ctx, window=16)
+    K = max(1, args.steps)
+    for r in d.run(K):
+        print(json.dumps({"stage": "round_driver", **dataclasses.asdict(r)}), flush=True)
+    # the library's launches of one round, timed on given logits (the logit generator is not the subject)
+    batch = synth.build_batch(cfg, "cuda")
+    p, out = d.p, d.out
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = ctx.kernel_launches()
+
+    def one(rnd):
+        p.round = rnd
+        ctx.mulo_sample_draft(p, batch["draft_lo"], d.tok_lo)
+        ctx.mulo_round(p, batch["cond"], batch["uncond"], batch["draft_lo"], d.tok_lo, batch["nn"],
+                       out["out_tok"], out["reject_bits"], out["expand_bits"], None, None, None,
+                       out["n_reject"], out["n_expand"], out["first_reject"])
+        ctx.mulo_islands(p, out["expand_bits"], d.labels, d.n_islands)
+        ctx.mulo_island_schedule(p, d.labels, d.window, d.step, d.n_steps)
+        ctx.mulo_downsample(p, out["out_tok"], d.prefix_lo)
+    for r in range(3):
+        one(r)
+    torch.cuda.synchronize()
+    n0 = ctx.kernel_launches()
+    e0.record()
+    for r in range(K):
+        one(3 + r)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / K
+    print(json.dumps({"stage": "round_driver", "metric": "rounds_per_sec", "value": 1e3 / ms, "unit": "rounds/s",
+                      "ms_per_round": ms, "steps": K, "gpu_launches_per_round": (ctx.kernel_launches() - n0) / K,
+                      "config": {"workload": workload_desc(cfg), "window": 16}, "data": "synthetic"}), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -601,6 +645,8 @@ def main():
                     help="time the rejection-island labelling of the workload's masks instead of the bench line")
     ap.add_argument("--draft-io", action="store_true",
                     help="time the drafter's sampling and the down-sampler stand-in instead of the bench line")
+    ap.add_argument("--driver", action="store_true",
+                    help="run the host loop over rounds (all stages, fresh synthetic logits per round)")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.workload]
     if args.batch:
@@ -611,6 +657,8 @@ def main():
         run_islands(args, cfg)
     elif args.draft_io:
         run_draft_io(args, cfg)
+    elif args.driver:
+        run_driver(args, cfg)
     elif args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -162,3 +162,24 @@ def test_limits_are_refused_before_launch(ctx):
     with pytest.raises(binding.MuloError) as e:
         ctx.mulo_islands(p, None, labels, n)
     assert e.value.status == binding.ERR_INVALID_ARG
+
+
+def test_round_driver_chains_the_stages(ctx):
+    """The host loop over rounds: every stage runs, the reports are consistent with the arrays behind them,
+    and the prefix for the next draft is the draft itself wherever nothing was redrawn."""
+    from paper_2601_05149_b200 import driver
+    cfg = synth.RoundConfig("drv", B=3, H=32, W=32, V=2048, dtype="bf16", top_k=256, cfg_scale=3.0, sigma=0.3,
+                            radius=1, seed=99)
+    d = driver.RoundDriver(cfg, ctx, window=4)
+    reports = d.run(3)
+    assert [r.round for r in reports] == [0, 1, 2]
+    assert len({r.acceptance_rate for r in reports}) > 1          # fresh logits every round
+    last = reports[-1]
+    assert 0.0 < last.acceptance_rate < 1.0 and last.redraw_fraction >= 1.0 - last.acceptance_rate
+    assert last.draft_steps == 4 * (cfg.h - 1) + cfg.w
+    labels, step = d.labels.cpu().numpy(), d.step.cpu().numpy()
+    expand = binding.unpack_bits(d.out["expand_bits"], cfg.W).numpy().astype(bool)
+    assert ((labels > 0) == expand).all() and ((step > 0) == expand).all()
+    assert last.target_steps_per_image == step.reshape(cfg.B, -1).max(1).sum() / cfg.B
+    untouched = expand.reshape(cfg.B, cfg.h, cfg.r, cfg.w, cfg.r).sum(axis=(2, 4)) == 0
+    assert (d.prefix_lo.cpu().numpy()[untouched] == d.tok_lo.cpu().numpy()[untouched]).all()
