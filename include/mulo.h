@@ -21,7 +21,9 @@
  *     workspace the caller hands to mulo_set_workspace.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls validate their arguments on the host, enqueue kernels on the stream
- *     and return; outputs are defined once the stream has been synchronised.
+ *     and return; outputs are defined once the stream has been synchronised.  Nothing a
+ *     call does blocks or leaves the stream, so calls can be captured into a CUDA graph
+ *     (parameters, `round` included, are frozen at capture) unless their text says otherwise.
  *   - Errors are return codes.  An invalid argument is detected before anything
  *     is launched.  Kernels never trap; contract violations they can see (a
  *     draft token with zero draft probability, a token id outside [0, V)) set a

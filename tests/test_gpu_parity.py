@@ -394,3 +394,38 @@ def test_pooling_on_the_streaming_path(ctx, scale, pool_k, delta):
     pooled = sum(int((o[b]["accept_prob"] > o[b]["p_tok"] / np.maximum(o[b]["q_tok"], 1e-300) * (1 + 1e-9)).sum())
                  for b in range(cfg.B))
     assert pooled > 0                                                 # some position did gain pooled mass
+
+
+def test_round_replays_from_a_cuda_graph(ctx):
+    """The calls only enqueue work on the given stream, so a round can be captured once and replayed."""
+    cfg = dataclasses.replace(synth.CONFIGS["C3"], name="graph", B=2, H=8, W=8, V=2048, top_k=250, radius=2,
+                              sigma=1.0, seed=77)
+    batch = pu.build_batch(cfg)
+    p = binding.params_from_config(cfg)
+    ctx.ensure_workspace(p)
+    direct = binding.alloc_round_outputs(p, "cuda", probs=True)
+    replay = binding.alloc_round_outputs(p, "cuda", probs=True)
+
+    def call(o):
+        ctx.mulo_round(p, batch["cond"], batch["uncond"], batch["draft_lo"], batch["tok_lo"], batch["nn"],
+                       o["out_tok"], o["reject_bits"], o["expand_bits"], o["p_tok"], o["q_tok"], o["accept_prob"],
+                       o["n_reject"], o["n_expand"], o["first_reject"])
+    call(direct)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        call(replay)                       # warm-up on the side stream, as graph capture wants
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call(replay)
+    for v in replay.values():
+        v.zero_()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    for k in direct:
+        assert torch.equal(direct[k], replay[k]), k
+    assert int(direct["n_reject"].sum()) > 0
