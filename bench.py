@@ -555,14 +555,14 @@ def run_draft_io(args, cfg):
                          "traffic": None},
             "cpu_baseline": cpu}), flush=True)
 
-    import oracle
-
     def orc_params(b):
+        import oracle
         return oracle.make_params(cfg.H, cfg.W, cfg.V, cfg.r, oracle.BF16 if cfg.dtype == "bf16" else oracle.F32,
                                   temperature=cfg.temperature, top_k=cfg.top_k, seed=cfg.seed, round=0, image=b)
     ms = timed(lambda: ctx.mulo_sample_draft(p, batch["draft_lo"], tok_lo))
     cpu = None
     if not args.no_cpu_baseline:
+        import oracle   # the CPU-baseline leg is the only user of the oracle here
         n_img = min(cfg.B, 2)
         t0 = time.time()
         for b in range(n_img):
@@ -575,6 +575,7 @@ def run_draft_io(args, cfg):
     ms = timed(lambda: ctx.mulo_downsample(p, tok_hi, tok_lo))
     cpu = None
     if not args.no_cpu_baseline:
+        import oracle
         x = tok_hi.cpu().numpy()
         t0 = time.time()
         for b in range(cfg.B):
