@@ -79,8 +79,10 @@
 
 /* borderline flags reported per position */
 #define ORC_FLAG_ACCEPT_EDGE 1u /* |u - thr| < 1e-6 (or pooled mass within 1e-6 rel. of tau) */
-#define ORC_FLAG_CDF_EDGE 2u    /* u' Z_w within 1e-6 (of mass) of an edge of the chosen CDF bin */
+#define ORC_FLAG_CDF_EDGE 2u    /* u' within 1e-6 of an edge of the chosen bin of the normalised CDF,
+                                   or a residual holding less than ORC_MIN_RESIDUAL_MASS      */
 #define ORC_FLAG_POOL_EDGE 4u   /* some prefix mass c_j within 1e-6 of delta          */
+#define ORC_MIN_RESIDUAL_MASS 1e-5
 
 typedef struct {
   int32_t H, W, V, r;
@@ -491,11 +493,12 @@ static void visit_position(const orc_params* P, const float* zt, const double* q
     t1 = orc_inverse_cdf(wts, V, u[1], &Zw, &eg);
   }
   out->tok_residual = t1;
-  /* The edge test of a draw is taken in units of probability mass, |u Z_w - C(x)| < 1e-6:
-   * the probabilities are only defined to the stated relative tolerance, so a
-   * residual that holds less than 1e-6 of mass decides nothing and is always
-   * borderline.  (Z_w = 1 for the target weights: there both readings agree.) */
-  out->flag_residual = eg * Zw < 1e-6 ? ORC_FLAG_CDF_EDGE : 0u;
+  /* A draw is borderline when its uniform lies within 1e-6 of an edge of the chosen bin of the
+   * NORMALISED CDF.  One more case: a residual that holds less than ORC_MIN_RESIDUAL_MASS of
+   * probability (target and draft all but equal) is rounding dust -- its shape is not defined
+   * at the precision of the probabilities themselves -- so every draw from it is borderline.
+   * (After the fall-back to the target weights Z_w = 1 and only the edge test applies.) */
+  out->flag_residual = (eg < 1e-6 || Zw < ORC_MIN_RESIDUAL_MASS) ? ORC_FLAG_CDF_EDGE : 0u;
   orc_residual_weights(p_prime, q, V, 0.0, wts);
   int t0 = orc_inverse_cdf(wts, V, u[2], &Zw, &eg);
   out->tok_target = t0;
