@@ -24,6 +24,9 @@
  *     and return; outputs are defined once the stream has been synchronised.  Nothing a
  *     call does blocks or leaves the stream, so calls can be captured into a CUDA graph
  *     (parameters, `round` included, are frozen at capture) unless their text says otherwise.
+ *   - A context is bound to one device.  Kernels are launched on the calling thread's
+ *     CURRENT device, so that device must be the context's: a call made while another
+ *     device is current returns MULO_ERR_INVALID_ARG before anything is enqueued.
  *   - Errors are return codes.  An invalid argument is detected before anything
  *     is launched.  Kernels never trap; contract violations they can see (a
  *     draft token with zero draft probability, a token id outside [0, V)) set a
@@ -304,7 +307,9 @@ mulo_status mulo_round_host(mulo_ctx* ctx, const mulo_params* p, void* arena, si
  *   - Size limit: mulo_workspace_bytes(p) must not exceed MULO_STATIC_SCRATCH_BYTES
  *     (about 80,000 grid positions per call, e.g. 19 images of 64 x 64).  A larger
  *     request returns MULO_ERR_WORKSPACE before anything is launched; split the batch
- *     over several calls (image_offset keeps the random streams aligned).
+ *     over several calls (image_offset keeps the random streams aligned).  Every other
+ *     refusal (a NULL or misaligned tensor, bad parameters, another device current)
+ *     also comes before the array is touched.
  *   - device_status [1], DEVICE pointer, may be NULL: receives the MULO_DEV_* bits this
  *     call raised (the call clears the bits first, so they describe this call alone).
  *   - The first call on a device looks up the array's device address (once per device, with

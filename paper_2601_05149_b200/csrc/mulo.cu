@@ -11,6 +11,7 @@
 #include "../../include/mulo.h"
 #include "mulo_dense.cuh"
 #include "mulo_islands.cuh"
+#include "mulo_lane.cuh"
 #include "mulo_stream.cuh"
 
 using namespace mulo;
@@ -460,6 +461,7 @@ struct mulo_ctx {
   std::vector<cudaEvent_t> ev;   // start/stop pairs around the fused row kernel
   size_t ev_used;
   int force_dense;               // diagnostics: never take the fast top-k path
+  int no_lane;                   // diagnostics: never take the lane-private kernel
 };
 
 static const size_t kStatusBytes = 256;
@@ -487,6 +489,18 @@ static mulo_status validate(const mulo_params* p) {
 }
 
 static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// Kernels are launched on the calling thread's current device, while limits, workspace and the
+// built-in scratch array belong to the context's device: the two must be the same.
+static mulo_status on_context_device(const mulo_ctx* ctx) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess) {
+    cudaGetLastError();
+    return MULO_ERR_CUDA;
+  }
+  return cur == ctx->device ? MULO_OK : MULO_ERR_INVALID_ARG;
+}
 
 static DevParams to_dev(const mulo_params* p) {
   DevParams d;
@@ -567,6 +581,7 @@ mulo_status mulo_create(mulo_ctx** out, int device) {
   c->launches = 0;
   c->ev_used = 0;
   c->force_dense = 0;
+  c->no_lane = 0;
   *out = c;
   return MULO_OK;
 }
@@ -764,7 +779,133 @@ static bool launch_stream(const mulo_ctx* ctx, const StreamArgs& s, size_t dyn, 
   return hu ? launch_stream_t<false, true>(ctx, s, dyn, st) : launch_stream_t<false, false>(ctx, s, dyn, st);
 }
 
+// ---- the lane-private fast path (V = 256 * W, W <= 64) ---------------------------------
+
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up once (host code only; no device work, no allocation).
+static TensorMapEncodeFn tensor_map_encoder() {
+  static std::once_flag once;
+  static TensorMapEncodeFn fn = nullptr;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (TensorMapEncodeFn)p;
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+// A logit tensor [rows, V] seen as [rows][256 threads][W ids]; one box = one phase of one row:
+// the next 32 bytes of every thread's id range, laid down with the 32-byte swizzle.
+static bool encode_row_map(CUtensorMap* tm, const void* base, size_t rows, int V, bool bf16) {
+  TensorMapEncodeFn enc = tensor_map_encoder();
+  if (!enc || rows == 0 || rows > 0xffffffffull) return false;
+  const int esz = bf16 ? 2 : 4, W = V / kLThreads;
+  const cuuint64_t gdim[3] = {(cuuint64_t)W, (cuuint64_t)kLThreads, (cuuint64_t)rows};
+  const cuuint64_t gstr[2] = {(cuuint64_t)W * esz, (cuuint64_t)V * esz};
+  const cuuint32_t box[3] = {(cuuint32_t)(32 / esz), (cuuint32_t)kLThreads, 1u};
+  const cuuint32_t es[3] = {1u, 1u, 1u};
+  return enc(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base),
+             gdim, gstr, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Fills `s` and returns the dynamic shared memory the lane kernel needs, or 0 if these
+// parameters are not eligible.
+static size_t plan_lane(const mulo_ctx* ctx, const DevParams& d, LaneArgs* s) {
+  if (d.top_k <= 0 || d.pool_k > 1) return 0;
+  const int V = d.V, k = d.top_k;
+  const int ids = d.bf16 ? 16 : 8;
+  if (V % (kLThreads * ids) != 0 || V / kLThreads > 64) return 0;
+  if (!tensor_map_encoder()) return 0;
+  // candidates aimed for beyond k: six standard deviations of the count of entries above a fixed
+  // value near the k-th largest (a row that comes up short is redone by the general routines, and
+  // even one such row costs more than the margin does)
+  const double p = (double)k / V;
+  const int margin = (int)fmax(64.0, 6.0 * sqrt(k * (1.0 - p)));
+  const int margin_boot = margin + 3 * margin / 4;   // rows without a prediction
+  if ((double)(k + margin_boot) > 0.5 * V) return 0;
+  // A list column serves two threads and holds four stacks (each thread's entries of the draft row
+  // and of the current target row): the bootstrap density's mean for 4 W ids plus six and a half
+  // standard deviations of that binomial count.  Three CTAs per SM are worth a somewhat shorter
+  // column (five and a half deviations).
+  const double pb = (double)(k + margin_boot) / V;
+  const double quad_mean = 4.0 * (V / kLThreads) * pb, quad_sd = sqrt(quad_mean * (1.0 - pb));
+  int R = (int)ceil(quad_mean + 6.5 * quad_sd) + 2;
+  if (R < 16) R = 16;
+  const size_t fixed = sizeof(LaneSmem) + 128 + 1024 + 256 + (size_t)kLStages * kLSlot;
+  const size_t per_cta3 = (size_t)228 * 1024 / 3;
+  if (per_cta3 > fixed) {
+    const int R3 = (int)((per_cta3 - fixed) / 512);
+    if (R3 < R && R3 >= (int)ceil(quad_mean + 5.5 * quad_sd) + 2) R = R3;
+  }
+  // one thread's own entries must fit the 32-bit mask of its low entries
+  if (0.25 * quad_mean + 6.5 * sqrt(0.25 * quad_mean * (1.0 - pb)) > 32.0) return 0;
+  const size_t dyn = 256 + (size_t)kLStages * kLSlot + (size_t)R * 512;
+  if (dyn + sizeof(LaneSmem) + 128 + 1024 > (size_t)ctx->smem_optin) return 0;
+  s->W = V / kLThreads;
+  s->n_ph = s->W / ids;
+  s->R = R;
+  s->margin = margin;
+  s->a_theta = (float)inv_norm_cdf(1.0 - p);
+  s->a_boot = (float)inv_norm_cdf(1.0 - (double)(k + margin_boot) / V);
+  s->a_max = (float)inv_norm_cdf(1.0 - 0.5 / V);
+  return dyn;
+}
+
+template <bool BF16, bool HAS_U>
+static bool launch_lane_t(const mulo_ctx* ctx, const LaneArgs& s, const CUtensorMap& tc, const CUtensorMap& tu,
+                          const CUtensorMap& tq, size_t dyn, cudaStream_t st) {
+  auto kern = k_round_lane<BF16, HAS_U>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kLThreads, dyn) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return false;
+  }
+  int grid = ctx->sm_count * per_sm;
+  if (grid > s.n_parents) grid = s.n_parents;
+  kern<<<grid, kLThreads, dyn, st>>>(s, tc, tu, tq);
+  return true;
+}
+
+static bool launch_lane(const mulo_ctx* ctx, const LaneArgs& s, size_t dyn, cudaStream_t st) {
+  const DevParams& d = s.P;
+  CUtensorMap tc, tu, tq;
+  const size_t rows = (size_t)d.B * d.H * d.W, cells = (size_t)d.B * d.h * d.w;
+  if (!encode_row_map(&tc, s.cond, rows, d.V, d.bf16)) return false;
+  if (!encode_row_map(&tu, s.uncond ? s.uncond : s.cond, rows, d.V, d.bf16)) return false;
+  if (!encode_row_map(&tq, s.draft, cells, d.V, d.bf16)) return false;
+  const bool hu = s.uncond != nullptr;
+  if (d.bf16) return hu ? launch_lane_t<true, true>(ctx, s, tc, tu, tq, dyn, st) : launch_lane_t<true, false>(ctx, s, tc, tu, tq, dyn, st);
+  return hu ? launch_lane_t<false, true>(ctx, s, tc, tu, tq, dyn, st) : launch_lane_t<false, false>(ctx, s, tc, tu, tq, dyn, st);
+}
+
 static size_t mask_smem(const mulo_params* p) { return (size_t)3 * p->H * ((p->W + 31) / 32) * 4; }
+
+// Everything mulo_round can refuse without touching the device.
+static mulo_status check_round_args(const mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond,
+                                    const void* tgt_uncond, const void* draft_logits_lo, const int32_t* draft_tok_lo,
+                                    const uint16_t* nn, const int32_t* out_tok, const uint32_t* reject_bits,
+                                    const uint32_t* expand_bits) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!tgt_cond || !draft_logits_lo || !draft_tok_lo || !out_tok || !reject_bits || !expand_bits)
+    return MULO_ERR_INVALID_ARG;
+  if (p->pool_k > 1 && !nn) return MULO_ERR_INVALID_ARG;
+  if (!aligned16(tgt_cond) || !aligned16(tgt_uncond) || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
+  return on_context_device(ctx);
+}
 
 extern "C" {
 
@@ -779,6 +920,7 @@ mulo_status mulo_upsample_pool(mulo_ctx* ctx, const mulo_params* p, const void* 
   if (!aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
   if (!ctx->ws) return MULO_ERR_WORKSPACE;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   RowKernelArgs a;
   memset(&a, 0, sizeof a);
   a.P = to_dev(p);
@@ -800,6 +942,7 @@ mulo_status mulo_island_schedule(mulo_ctx* ctx, const mulo_params* p, const int3
   if (!labels || !step || !n_steps || window < 1) return MULO_ERR_INVALID_ARG;
   if ((size_t)p->H * p->W > (size_t)kIslandMaxCells) return MULO_ERR_UNSUPPORTED;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   ScheduleArgs a;
   a.H = p->H; a.W = p->W; a.window = window > p->W ? p->W : window;
   a.labels = labels; a.step = step; a.n_steps = n_steps;
@@ -821,6 +964,7 @@ mulo_status mulo_sample_draft(mulo_ctx* ctx, const mulo_params* p, const void* d
   if (!draft_logits_lo || !draft_tok_lo || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
   if (!ctx->ws) return MULO_ERR_WORKSPACE;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   RowKernelArgs a;
   memset(&a, 0, sizeof a);
@@ -861,6 +1005,7 @@ mulo_status mulo_downsample(mulo_ctx* ctx, const mulo_params* p, const int32_t* 
   if (!tok_hi || !tok_lo) return MULO_ERR_INVALID_ARG;
   if (p->r > 16) return MULO_ERR_UNSUPPORTED;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   const int h = p->H / p->r, w = p->W / p->r, cells = p->B * h * w;
   k_downsample<<<(cells + 255) / 256, 256, 0, (cudaStream_t)stream>>>(tok_hi, tok_lo, cells, h, w, p->W, p->r);
   return launched(ctx, 1);
@@ -882,6 +1027,7 @@ mulo_status mulo_verify(mulo_ctx* ctx, const mulo_params* p, const void* tgt_con
   Workspace w;
   if ((s = check_ws(ctx, p, &w)) != MULO_OK) return s;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   RowKernelArgs a;
   memset(&a, 0, sizeof a);
   a.P = to_dev(p);
@@ -915,6 +1061,7 @@ mulo_status mulo_local_reject_expand(mulo_ctx* ctx, const mulo_params* p, const 
   if (s != MULO_OK) return s;
   if (!reject_bits || !first_reject || !expand_bits || !n_expand) return MULO_ERR_INVALID_ARG;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   MaskArgs m;
   memset(&m, 0, sizeof m);
   m.H = p->H; m.W = p->W; m.r = p->r; m.radius = p->radius; m.clip = p->clip_before_first != 0;
@@ -934,6 +1081,7 @@ mulo_status mulo_islands(mulo_ctx* ctx, const mulo_params* p, const uint32_t* ex
   if (!expand_bits || !labels || !n_islands || max_islands < 0) return MULO_ERR_INVALID_ARG;
   if ((size_t)p->H * p->W > (size_t)kIslandMaxCells) return MULO_ERR_UNSUPPORTED;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   IslandArgs a;
   a.H = p->H; a.W = p->W; a.max_islands = max_islands;
   a.bits = expand_bits; a.labels = labels; a.n_islands = n_islands;
@@ -963,6 +1111,7 @@ mulo_status mulo_resample(mulo_ctx* ctx, const mulo_params* p, const void* tgt_c
   if (!aligned16(tgt_cond) || !aligned16(tgt_uncond) || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
   if (!ctx->ws) return MULO_ERR_WORKSPACE;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   RowKernelArgs a;
   memset(&a, 0, sizeof a);
   a.P = to_dev(p);
@@ -987,13 +1136,9 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
                        int32_t* out_tok, uint32_t* reject_bits, uint32_t* expand_bits, float* p_tok,
                        float* q_tok, float* accept_prob, int32_t* n_reject, int32_t* n_expand,
                        int32_t* first_reject, void* stream) {
-  if (!ctx) return MULO_ERR_INVALID_ARG;
-  mulo_status s = validate(p);
+  mulo_status s = check_round_args(ctx, p, tgt_cond, tgt_uncond, draft_logits_lo, draft_tok_lo, nn, out_tok,
+                                   reject_bits, expand_bits);
   if (s != MULO_OK) return s;
-  if (!tgt_cond || !draft_logits_lo || !draft_tok_lo || !out_tok || !reject_bits || !expand_bits)
-    return MULO_ERR_INVALID_ARG;
-  if (p->pool_k > 1 && !nn) return MULO_ERR_INVALID_ARG;
-  if (!aligned16(tgt_cond) || !aligned16(tgt_uncond) || !aligned16(draft_logits_lo)) return MULO_ERR_INVALID_ARG;
   Workspace w;
   if ((s = check_ws(ctx, p, &w)) != MULO_OK) return s;
   if (p->B == 0) return MULO_OK;
@@ -1014,10 +1159,25 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   cudaStream_t st = (cudaStream_t)stream;
   const bool timed = ctx->ev_used + 2 <= ctx->ev.size();
   if (timed) cudaEventRecord(ctx->ev[ctx->ev_used], st);
+  bool fast = false;
+  LaneArgs la;
+  memset(&la, 0, sizeof la);
+  const size_t ldyn = (ctx->force_dense || ctx->no_lane) ? 0 : plan_lane(ctx, a.P, &la);
+  if (ldyn) {
+    la.P = a.P;
+    la.cond = a.cond; la.uncond = a.uncond; la.draft = a.draft; la.draft_tok_lo = draft_tok_lo;
+    la.p_tok = p_tok; la.q_tok = q_tok; la.accept_prob = accept_prob;
+    la.flags = w.flags; la.cand_res = w.cand_res; la.cand_tgt = w.cand_tgt;
+    la.dev_status = w.status;
+    la.fail_list = w.fail_list;
+    la.n_parents = p->B * a.P.h * a.P.w;
+    if (cudaMemsetAsync(w.status + kFailCount, 0, sizeof(uint32_t), st) != cudaSuccess) return MULO_ERR_CUDA;
+    fast = launch_lane(ctx, la, ldyn, st);
+    if (fast) k_verify_failed<<<2 * ctx->sm_count, kThreads, dyn, st>>>(a, w.fail_list, w.status + kFailCount);
+  }
   StreamArgs sa;
   memset(&sa, 0, sizeof sa);
-  const size_t sdyn = ctx->force_dense ? 0 : plan_stream(ctx, a.P, &sa);
-  bool fast = false;
+  const size_t sdyn = (ctx->force_dense || fast) ? 0 : plan_stream(ctx, a.P, &sa);
   if (sdyn) {
     sa.P = a.P;
     sa.cond = a.cond; sa.uncond = a.uncond; sa.draft = a.draft; sa.draft_tok_lo = draft_tok_lo;
@@ -1100,6 +1260,7 @@ mulo_status mulo_round_host(mulo_ctx* ctx, const mulo_params* p, void* arena, si
   const HostArena A = carve_arena(p, tgt_uncond != nullptr);
   if (A.total > arena_bytes) return MULO_ERR_WORKSPACE;
   if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
   char* d = (char*)arena;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t n = (size_t)p->B * p->H * p->W, nlo = n / ((size_t)p->r * p->r);
@@ -1179,8 +1340,9 @@ extern "C" mulo_status mulo_round_static(mulo_ctx* ctx, const mulo_params* p, co
                                          float* q_tok, float* accept_prob, int32_t* n_reject,
                                          int32_t* n_expand, int32_t* first_reject, uint32_t* device_status,
                                          void* stream) {
-  if (!ctx) return MULO_ERR_INVALID_ARG;
-  mulo_status s = validate(p);
+  // every refusal comes before the shared array is touched
+  mulo_status s = check_round_args(ctx, p, tgt_cond, tgt_uncond, draft_logits_lo, draft_tok_lo, nn, out_tok,
+                                   reject_bits, expand_bits);
   if (s != MULO_OK) return s;
   if (carve_ws(nullptr, p).bytes > (size_t)MULO_STATIC_SCRATCH_BYTES) return MULO_ERR_WORKSPACE;
   void* scratch = nullptr;

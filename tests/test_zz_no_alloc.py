@@ -73,6 +73,8 @@ def test_static_scratch_round_equals_workspace_round():
     _static_round(ctx, small, b2, status)
     assert int(status.item()) == 0
 
+    o_big = binding.alloc_round_outputs(binding.params_from_config(big), "cuda", False)   # before the memory reading below
+
     # a request beyond the array is refused before anything is launched
     huge = binding.make_params(32, 64, 64, 4096, 2, binding.BF16)
     assert binding.Context.workspace_bytes(huge) > binding.STATIC_SCRATCH_BYTES
@@ -81,5 +83,30 @@ def test_static_scratch_round_equals_workspace_round():
     with pytest.raises(binding.MuloError) as e:
         ctx.mulo_round_static(huge, b1["cond"], None, b1["draft_lo"], b1["tok_lo"], None, dummy, dummy, dummy)
     assert e.value.status == binding.ERR_WORKSPACE and ctx.kernel_launches() == launches
+
+    # an invalid argument (a misaligned tensor, a missing output) is refused before anything is
+    # enqueued, the clearing of the shared array's status word included
+    p2 = binding.params_from_config(small)
+    o = binding.alloc_round_outputs(p2, "cuda", False)
+    skewed = torch.empty(b2["cond"].numel() + 4, dtype=b2["cond"].dtype, device="cuda")[1:1 + b2["cond"].numel()]
+    assert skewed.data_ptr() % 16 != 0
+    launches = ctx.kernel_launches()
+    with pytest.raises(binding.MuloError) as e:
+        ctx.mulo_round_static(p2, skewed.view(b2["cond"].shape), None, b2["draft_lo"], b2["tok_lo"], b2["nn"],
+                              o["out_tok"], o["reject_bits"], o["expand_bits"])
+    assert e.value.status == binding.ERR_INVALID_ARG and ctx.kernel_launches() == launches
+    with pytest.raises(binding.MuloError):
+        ctx.mulo_round_static(p2, b2["cond"], None, b2["draft_lo"], b2["tok_lo"], b2["nn"], None,
+                              o["reject_bits"], o["expand_bits"])
+
+    # the call allocates nothing: free device memory is the same before and after warmed-up calls
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for rnd in range(3):
+        ctx.mulo_round_static(binding.params_from_config(big, round=rnd), b1["cond"], b1["uncond"], b1["draft_lo"],
+                              b1["tok_lo"], b1["nn"], o_big["out_tok"], o_big["reject_bits"], o_big["expand_bits"])
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
     ref_ctx.close()
     ctx.close()
