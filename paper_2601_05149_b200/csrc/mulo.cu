@@ -801,15 +801,16 @@ static TensorMapEncodeFn tensor_map_encoder() {
   return fn;
 }
 
-// A logit tensor [rows, V] seen as [rows][256 threads][W ids]; one box = one phase of one row:
-// the next 32 bytes of every thread's id range, laid down with the 32-byte swizzle.
+// A logit tensor [rows, V] seen as [rows][256 threads][W ids]; one box = one phase of one warp's
+// part of a row: the next 32 bytes of the id range of each of its 32 lanes, laid down with the
+// 32-byte swizzle.
 static bool encode_row_map(CUtensorMap* tm, const void* base, size_t rows, int V, bool bf16) {
   TensorMapEncodeFn enc = tensor_map_encoder();
   if (!enc || rows == 0 || rows > 0xffffffffull) return false;
   const int esz = bf16 ? 2 : 4, W = V / kLThreads;
   const cuuint64_t gdim[3] = {(cuuint64_t)W, (cuuint64_t)kLThreads, (cuuint64_t)rows};
   const cuuint64_t gstr[2] = {(cuuint64_t)W * esz, (cuuint64_t)V * esz};
-  const cuuint32_t box[3] = {(cuuint32_t)(32 / esz), (cuuint32_t)kLThreads, 1u};
+  const cuuint32_t box[3] = {(cuuint32_t)(32 / esz), 32u, 1u};   // one warp's lanes
   const cuuint32_t es[3] = {1u, 1u, 1u};
   return enc(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base),
              gdim, gstr, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
@@ -836,18 +837,29 @@ static size_t plan_lane(const mulo_ctx* ctx, const DevParams& d, LaneArgs* s) {
   // standard deviations of that binomial count.  Three CTAs per SM are worth a somewhat shorter
   // column (five and a half deviations).
   const double pb = (double)(k + margin_boot) / V;
-  const double quad_mean = 4.0 * (V / kLThreads) * pb, quad_sd = sqrt(quad_mean * (1.0 - pb));
-  int R = (int)ceil(quad_mean + 6.5 * quad_sd) + 2;
+  const double mu = (double)(V / kLThreads) * pb, var = mu * (1.0 - pb);   // entries of one thread in one row
+  const double quad_mean = 4.0 * mu, quad_sd = sqrt(4.0 * var);
+  // ... and a thread stops appending when fewer rows than one phase's ids are left before the other
+  // thread's stack, so the column must also hold both draft stacks, what the thread has gathered
+  // by its last phase, and one more phase
+  const int n_ph = (V / kLThreads) / ids;
+  const double part = (double)(n_ph - 1) / n_ph;
+  auto rows_needed = [&](double dev) {
+    const double a1 = quad_mean + dev * quad_sd + 2.0;
+    const double a2 = (2.0 + part) * mu + dev * sqrt(var * (2.0 + part * part)) + ids + 2.0;
+    return (int)ceil(fmax(a1, a2));
+  };
+  int R = rows_needed(6.5);
   if (R < 16) R = 16;
-  const size_t fixed = sizeof(LaneSmem) + 128 + 1024 + 256 + (size_t)kLStages * kLSlot;
+  const size_t fixed = sizeof(LaneSmem) + 128 + 1024 + 256 + (size_t)kLRing;
   const size_t per_cta3 = (size_t)228 * 1024 / 3;
   if (per_cta3 > fixed) {
     const int R3 = (int)((per_cta3 - fixed) / 512);
-    if (R3 < R && R3 >= (int)ceil(quad_mean + 5.5 * quad_sd) + 2) R = R3;
+    if (R3 < R && R3 >= rows_needed(5.5)) R = R3;
   }
   // one thread's own entries must fit the 32-bit mask of its low entries
   if (0.25 * quad_mean + 6.5 * sqrt(0.25 * quad_mean * (1.0 - pb)) > 32.0) return 0;
-  const size_t dyn = 256 + (size_t)kLStages * kLSlot + (size_t)R * 512;
+  const size_t dyn = 256 + (size_t)kLRing + (size_t)R * 512;
   if (dyn + sizeof(LaneSmem) + 128 + 1024 > (size_t)ctx->smem_optin) return 0;
   s->W = V / kLThreads;
   s->n_ph = s->W / ids;

@@ -2,12 +2,14 @@
 // evenly over a CTA's 256 threads (V = 256 * W, W <= 64 ids per thread).
 //
 // A persistent CTA (256 threads, three per SM) owns a contiguous range of parent (low-res)
-// cells.  Per parent it streams the draft row and then its r*r target rows ONCE through a
-// two-slot shared-memory ring.  A slot holds one PHASE of a row: a tiled bulk-tensor copy
-// (never multicast) brings 32 bytes for every thread -- the next 16 bf16 (8 fp32) ids of
-// the 64-id range that thread owns -- of the conditional and of the unconditional row,
-// placed with the 32-byte swizzle so that the 128-bit shared loads of a quarter warp hit
-// eight different bank groups.  Owning a CONTIGUOUS id range is what keeps the rest cheap:
+// cells.  Per parent it streams the draft row and then its r*r target rows ONCE.  Every WARP has
+// a two-slot shared-memory ring of its own: a slot holds one PHASE of the warp's part of a row,
+// brought by a tiled bulk-tensor copy (never multicast) -- 32 bytes for every lane, the next
+// 16 bf16 (8 fp32) ids of the 64-id range that thread owns, of the conditional and of the
+// unconditional row, placed with the 32-byte swizzle so that the 128-bit shared loads of a
+// quarter warp hit eight different bank groups.  A warp waits for its own data only and requests
+// its next phase itself, the moment the slot's words are in registers; the warps of a CTA meet
+// at the row's first block barrier.  Owning a CONTIGUOUS id range is what keeps the rest cheap:
 //
 //   dense phase   per element: unpack, CFG mix (packed fp32, one IEEE rounding per step),
 //                 compare with a predicted pivot, and a predicated append of the survivor
@@ -46,8 +48,10 @@ namespace mulo {
 constexpr int kLThreads = 256;
 constexpr int kLWarps = kLThreads / 32;
 constexpr int kLStages = 2;
-constexpr int kLTile = kLThreads * 32;   // bytes of one tensor's tile: 32 bytes per thread
+constexpr int kLTile = 32 * 32;          // bytes of one tensor's tile of one warp: 32 bytes per lane
 constexpr int kLSlot = 2 * kLTile;       // conditional + unconditional
+constexpr int kLWarpRing = kLStages * kLSlot;   // ring bytes of one warp
+constexpr int kLRing = kLWarps * kLWarpRing;    // ring bytes of the CTA
 constexpr int kLBins = 256;
 constexpr int kLSetAside = 64;           // entries of the crossing bin that are ranked exactly
 constexpr float kLog2e = 1.4426950408889634f;
@@ -86,19 +90,21 @@ struct LanePredictor {
   int dir;
 };
 
-struct LaneCursor {            // next item to request into a ring slot
-  int left;                    // items still to request into this slot
+struct LaneCursor {            // next item a warp requests into its ring (phases in consumption order)
+  int left;                    // items still to request
   int ph, j;                   // phase within the row, row within the parent (0 = draft row)
-  int parent, b, ca, cc;
+  int parent;
 };
+constexpr int kLMaxRows = 17;  // draft row + r*r children, r <= 4
 
 // Selection scratch of one row.  Two copies, used by rows of alternating parity: what a row adds
 // into (histogram, set-aside list, per-warp partials) is reset / rewritten two rows later, with
 // at least two block barriers in between, so no reader of row i can meet a writer of row i + 2.
 struct LaneSel {
-  unsigned hist[kLBins];
+  alignas(16) unsigned hist[kLBins];
   float sa_z[kLSetAside];
   float sa_e[kLSetAside];
+  unsigned short sa_owner[kLSetAside];   // the thread whose list holds the entry
   unsigned n_sa;
   unsigned overflow;
   int w_n[kLWarps];
@@ -115,9 +121,8 @@ struct LanePrep {              // per target row, written by two threads before 
 };
 
 struct LaneSmem {
-  uint64_t full[kLStages];
-  unsigned done[kLStages];
-  LaneCursor cursor[kLStages];
+  uint64_t full[kLWarps][kLStages];   // every warp has a ring of its own
+  LaneCursor cursor[kLWarps];
   LaneSel sel[2];
   LanePrep prep[2];
   double w_tot[2][kLWarps];    // block scan of a draw; consecutive draws alternate
@@ -127,6 +132,8 @@ struct LaneSmem {
   double q_tok;                // of the current parent
   uint32_t raw_q;              // landing place of the draft logit word of x~
   int tok[2];                  // the draft token of the parent in work / of the next one
+  int rows[2][kLMaxRows];      // row index (within its tensor) of every row of a parent, by parent parity
+  int image[2];                // image index of the parent, by parent parity
 };
 
 __device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint64_t* bar) {
@@ -135,24 +142,12 @@ __device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap* tm,
       "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
       : "memory");
 }
-// Bounded wait on a ring slot.  The hint lets the hardware suspend the warp for up to about a
-// microsecond per try instead of spinning through the issue slots; after 2^21 tries (seconds) the
-// wait gives up and raises the time-out bit.
-__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
-      : "memory");
-  return ok != 0;
-}
+// Bounded wait on a ring slot: after kSpinLimit tries the wait gives up and raises the time-out bit.
 __device__ __forceinline__ void lane_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status) {
+  if (mbar_try_wait(bar, parity)) return;
 #pragma unroll 1
-  for (uint32_t it = 0; it < (1u << 21); ++it)
-    if (mbar_try_wait_hint(bar, parity, 1000u)) return;
+  for (uint32_t it = 0; it < kSpinLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return;
   atomicOr(dev_status, MULO_DEV_TIMEOUT);
 }
 // 4-byte asynchronous global -> shared copy (no register holds the value while it is in flight)
@@ -190,16 +185,21 @@ __device__ __forceinline__ float ex2f(float t) {
   return r;
 }
 
-// Appends z to a thread's list if z >= pivot, without a branch: the store is unconditional (a
-// value below the pivot lands in the next free row and is overwritten by the next survivor, or
-// never read), the cursor steps -- clamped at `lim` -- and the mask gains the bit under a select.
-template <int STEP, int BIT>
-__device__ __forceinline__ void lane_put(float z, float pivot, uint32_t& cur, uint32_t lim, uint32_t& m) {
-  const bool p = z >= pivot;
-  sts_f32(cur, z);
-  const uint32_t nxt = STEP > 0 ? min(cur + (uint32_t)STEP, lim) : max(cur - (uint32_t)(-STEP), lim);
-  cur = p ? nxt : cur;
-  m |= p ? (1u << BIT) : 0u;
+// Appends z to a thread's list if z >= pivot: four instructions -- compare, store, cursor step,
+// the survivor's bit in the mask -- the last three predicated.  Written in PTX: left to the
+// compiler, the same statements become a branch and several moves per element.  `stp` is the
+// thread's step (+-512 bytes, or 0 once its column has no room left for a whole phase).
+template <int BIT>
+__device__ __forceinline__ void lane_put(float z, float pivot, uint32_t& cur, uint32_t stp, uint32_t& m) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ge.f32 p, %2, %3;\n\t"
+      "@p st.shared.f32 [%0], %2;\n\t"
+      "@p add.u32 %0, %0, %4;\n\t"
+      "@p or.b32 %1, %1, %5;\n\t}"
+      : "+r"(cur), "+r"(m)
+      : "f"(z), "f"(pivot), "r"(stp), "n"(1u << BIT)
+      : "memory");
 }
 
 template <int J>
@@ -210,58 +210,133 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v) {
 // Two ids of a phase: word J of 16-byte piece I of the thread's 32 bytes.  bf16: one word of the
 // conditional (and unconditional) row holds both; fp32: words 2J and 2J + 1 of piece I hold them
 // (J < 2).  Pre-processing as the definition says (d = c - u; v = fma(s, d, u); z = v * invT, each
-// one fp32 rounding; two ids per instruction), then the two appends.
-template <bool BF16, bool ROW_U, bool SCALE, int STEP, int I, int J>
-__device__ __forceinline__ void lane_pair(const uint4 (&c)[2], const uint4 (&u)[2], uint64_t s2, uint64_t t2,
-                                          float pivot, uint32_t& cur, uint32_t lim, uint32_t& m) {
-  uint64_t v, un;
+// one fp32 rounding; two ids per packed instruction), then the two appends.
+template <bool BF16, bool ROW_U, bool SCALE, int I, int J>
+__device__ __forceinline__ void lane_pair(const uint4 (&c)[2], const uint4 (&u)[2], float2 s2, float2 t2,
+                                          float pivot, uint32_t& cur, uint32_t stp, uint32_t& m) {
+  float2 v, un;
   if (BF16) {
     const uint32_t cw = word_of<J>(c[I]);
-    v = pack2(bf16_lo(cw), bf16_hi(cw));
+    v = make_float2(bf16_lo(cw), bf16_hi(cw));
     if (ROW_U) {
       const uint32_t uw = word_of<J>(u[I]);
-      un = pack2(bf16_lo(uw), bf16_hi(uw));
+      un = make_float2(bf16_lo(uw), bf16_hi(uw));
     }
   } else {
-    v = pack2(__uint_as_float(word_of<(2 * J) & 3>(c[I])), __uint_as_float(word_of<(2 * J + 1) & 3>(c[I])));
-    if (ROW_U) un = pack2(__uint_as_float(word_of<(2 * J) & 3>(u[I])), __uint_as_float(word_of<(2 * J + 1) & 3>(u[I])));
+    v = make_float2(__uint_as_float(word_of<(2 * J) & 3>(c[I])), __uint_as_float(word_of<(2 * J + 1) & 3>(c[I])));
+    if (ROW_U)
+      un = make_float2(__uint_as_float(word_of<(2 * J) & 3>(u[I])), __uint_as_float(word_of<(2 * J + 1) & 3>(u[I])));
   }
-  if (ROW_U) v = fma2(s2, sub2(v, un), un);
-  if (SCALE) v = mul2(v, t2);
-  float z0, z1;
-  unpack2(v, z0, z1);
+  if (ROW_U) v = __ffma2_rn(s2, __ffma2_rn(un, make_float2(-1.f, -1.f), v), un);   // fma(u, -1, c) rounds as c - u
+  if (SCALE) v = __fmul2_rn(v, t2);
   constexpr int bit = BF16 ? I * 8 + J * 2 : I * 4 + J * 2;
-  lane_put<STEP, bit>(z0, pivot, cur, lim, m);
-  lane_put<STEP, bit + 1>(z1, pivot, cur, lim, m);
+  lane_put<bit>(v.x, pivot, cur, stp, m);
+  lane_put<bit + 1>(v.y, pivot, cur, stp, m);
 }
 
-// One phase of a row for one thread: the 32 bytes (16 bf16 / 8 fp32 ids) of the conditional row at
-// `sb` (and of the unconditional row one tile further); survivors z >= pivot are appended at `cur`
+// One phase of a row for one thread, in two steps.  lane_load: the 32 bytes (16 bf16 / 8 fp32 ids)
+// of the conditional row at `sb` and of the unconditional row one tile further, into registers
+// (after which the slot can be refilled).  lane_dense: survivors z >= pivot are appended at `cur`
 // (stepping by STEP bytes, clamped at `lim`) and marked in the returned mask.
-template <bool BF16, bool ROW_U, bool SCALE, int STEP>
-__device__ __forceinline__ uint32_t lane_dense(uint32_t sb, uint32_t sw, float s, float invT, float pivot,
-                                               uint32_t& cur, uint32_t lim) {
-  // the second 16 bytes are loaded after the first have been worked off: half as many live registers
-  uint4 c[2], u[2];
-  c[0] = lds128(sb + (sw << 4));
-  u[0] = ROW_U ? lds128(sb + kLTile + (sw << 4)) : make_uint4(0, 0, 0, 0);
-  const uint64_t s2 = pack2(s, s), t2 = pack2(invT, invT);
-  uint32_t m = 0;
-  lane_pair<BF16, ROW_U, SCALE, STEP, 0, 0>(c, u, s2, t2, pivot, cur, lim, m);
-  lane_pair<BF16, ROW_U, SCALE, STEP, 0, 1>(c, u, s2, t2, pivot, cur, lim, m);
-  if (BF16) {
-    lane_pair<BF16, ROW_U, SCALE, STEP, 0, 2>(c, u, s2, t2, pivot, cur, lim, m);
-    lane_pair<BF16, ROW_U, SCALE, STEP, 0, 3>(c, u, s2, t2, pivot, cur, lim, m);
+template <bool ROW_U>
+__device__ __forceinline__ void lane_load(uint32_t sb, uint32_t sw, uint4 (&c)[2], uint4 (&u)[2]) {
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    c[i] = lds128(sb + (((uint32_t)i ^ sw) << 4));
+    u[i] = ROW_U ? lds128(sb + kLTile + (((uint32_t)i ^ sw) << 4)) : make_uint4(0, 0, 0, 0);
   }
-  c[1] = lds128(sb + ((1u ^ sw) << 4));
-  u[1] = ROW_U ? lds128(sb + kLTile + ((1u ^ sw) << 4)) : make_uint4(0, 0, 0, 0);
-  lane_pair<BF16, ROW_U, SCALE, STEP, 1, 0>(c, u, s2, t2, pivot, cur, lim, m);
-  lane_pair<BF16, ROW_U, SCALE, STEP, 1, 1>(c, u, s2, t2, pivot, cur, lim, m);
+}
+template <bool BF16, bool ROW_U, bool SCALE>
+__device__ __forceinline__ uint32_t lane_dense(const uint4 (&c)[2], const uint4 (&u)[2], float s, float invT,
+                                               float pivot, uint32_t& cur, uint32_t stp) {
+  const float2 s2 = make_float2(s, s), t2 = make_float2(invT, invT);
+  uint32_t m = 0;
+  lane_pair<BF16, ROW_U, SCALE, 0, 0>(c, u, s2, t2, pivot, cur, stp, m);
+  lane_pair<BF16, ROW_U, SCALE, 0, 1>(c, u, s2, t2, pivot, cur, stp, m);
   if (BF16) {
-    lane_pair<BF16, ROW_U, SCALE, STEP, 1, 2>(c, u, s2, t2, pivot, cur, lim, m);
-    lane_pair<BF16, ROW_U, SCALE, STEP, 1, 3>(c, u, s2, t2, pivot, cur, lim, m);
+    lane_pair<BF16, ROW_U, SCALE, 0, 2>(c, u, s2, t2, pivot, cur, stp, m);
+    lane_pair<BF16, ROW_U, SCALE, 0, 3>(c, u, s2, t2, pivot, cur, stp, m);
+  }
+  lane_pair<BF16, ROW_U, SCALE, 1, 0>(c, u, s2, t2, pivot, cur, stp, m);
+  lane_pair<BF16, ROW_U, SCALE, 1, 1>(c, u, s2, t2, pivot, cur, stp, m);
+  if (BF16) {
+    lane_pair<BF16, ROW_U, SCALE, 1, 2>(c, u, s2, t2, pivot, cur, stp, m);
+    lane_pair<BF16, ROW_U, SCALE, 1, 3>(c, u, s2, t2, pivot, cur, stp, m);
   }
   return m;
+}
+
+// 2^x in double, out of line: three call sites, a few hundred instructions each otherwise
+__device__ __noinline__ double lane_exp2(double x) { return exp2(x); }
+
+// Philox4x32-10 as a rolled loop (one thread per row runs it; the unrolled form is ten times the code)
+__device__ __noinline__ uint4 lane_philox(uint4 c, uint2 k) {
+#pragma unroll 1
+  for (int i = 0; i < 10; ++i) {
+    const uint32_t a = 0xD2511F53u, b = 0xCD9E8D57u;
+    const uint32_t h0 = __umulhi(a, c.x), l0 = a * c.x;
+    const uint32_t h1 = __umulhi(b, c.z), l1 = b * c.z;
+    c = make_uint4(h1 ^ c.y ^ k.x, l1, h0 ^ c.w ^ k.y, l0);
+    k.x += 0x9E3779B9u;
+    k.y += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// The optional probability outputs of a position (one thread; out of line: double divisions).
+__device__ __noinline__ void lane_write_probs(float* p_tok, float* q_tok_out, float* accept_prob, size_t g, double e_tok,
+                                              double q_tok, double Z, bool threshold_rule) {
+  const double p = e_tok / Z;
+  if (p_tok) p_tok[g] = (float)p;
+  if (q_tok_out) q_tok_out[g] = (float)q_tok;
+  if (accept_prob) {
+    double thr;
+    if (threshold_rule) thr = p;
+    else if (q_tok <= 0.0) thr = p > 0.0 ? 1.0 : 0.0;
+    else thr = fmin(1.0, p / q_tok);
+    accept_prob[g] = (float)thr;
+  }
+}
+
+// The predictor of one kind of row after a row (ok: theta found exactly).  One thread; out of line.
+__device__ __noinline__ void lane_learn(LanePredictor* prp, bool ok, int reason, float theta, float pivot, int n,
+                                        int n_ge, float mx, int margin, float a_theta, float a_boot) {
+  LanePredictor pr = *prp;
+  if (!ok) {
+    pr.have = 0;
+    const int dir = reason == 2 ? -1 : (reason == 1 || reason == 3) ? 1 : 0;
+    if (dir != 0) {
+      const float unit = 0.5f * (a_theta - a_boot);
+      if (pr.dir == 0) pr.step = unit;
+      else if (pr.dir == dir) pr.step = fminf(2.0f * pr.step, 64.0f * unit);
+      else pr.step = fmaxf(0.5f * pr.step, 0.25f * unit);
+      pr.shift += (float)dir * pr.step;
+      pr.dir = dir;
+    }
+  } else {
+    pr.dir = 0;
+    const int below = n - n_ge;   // candidates in [pivot, theta)
+    float rho = pr.rho;
+    bool rho_ok = pr.have != 0;
+    if (theta > pivot && below >= 16) {
+      const float r_new = (float)below / (theta - pivot);
+      rho = pr.have ? pr.rho + 0.25f * (r_new - pr.rho) : r_new;
+      rho_ok = true;
+    }
+    if (!rho_ok) {
+      pr.have = 0;
+    } else {
+      pr.theta = pr.have ? pr.theta + 0.25f * (theta - pr.theta) : theta;
+      pr.mx = pr.have ? pr.mx + 0.25f * (mx - pr.mx) : mx;
+      pr.rho = rho;
+      pr.have = 1;
+      const float d = (float)margin / rho;
+      pr.pivot = pr.theta - d;
+      pr.inv_w = (float)kLBins / (2.0f * d);   // the histogram spans twice the distance pivot -> threshold
+      pr.ref = pr.mx;
+    }
+  }
+  *prp = pr;
 }
 
 template <bool BF16, bool HAS_U>
@@ -293,17 +368,16 @@ __global__ void __launch_bounds__(kLThreads, 3)
   // of the other thread; whether two stacks met is checked from the four counts.
   const bool up = tid < kLThreads / 2;
   const int step = up ? 512 : -512;
-  const uint32_t col = ring + kLStages * kLSlot + (uint32_t)(tid & 127) * 4u;
+  const uint32_t col = ring + kLRing + (uint32_t)(tid & 127) * 4u;
   const uint32_t q_base = col + (up ? 0u : (uint32_t)(R - 1) * 512u);
   const uint32_t q_lim = col + (up ? (uint32_t)(R - 1) * 512u : 0u);   // the partner's first draft row
-  const uint32_t sw = ((uint32_t)tid >> 2) & 1u;           // 32-byte swizzle: address bit 4 ^= bit 7
-  const uint32_t my_off = (uint32_t)tid * 32u;
+  const uint32_t sw = ((uint32_t)lane >> 2) & 1u;          // 32-byte swizzle: address bit 4 ^= bit 7
+  const uint32_t wring = ring + (uint32_t)warp * kLWarpRing;   // this warp's ring
+  const uint32_t my_off = (uint32_t)lane * 32u;
 
   if (tid == 0) {
-    for (int s = 0; s < kLStages; ++s) {
-      mbar_init(&sm.full[s], 1);
-      sm.done[s] = 0;
-    }
+    for (int w = 0; w < kLWarps; ++w)
+      for (int s = 0; s < kLStages; ++s) mbar_init(&sm.full[w][s], 1);
     mbar_fence_init();
     for (int s = 0; s < 2; ++s) {
       sm.sel[s].n_sa = 0;
@@ -319,113 +393,108 @@ __global__ void __launch_bounds__(kLThreads, 3)
   sm.sel[1].hist[tid] = 0;
   __syncthreads();
 
-  // ---- the ring: items in the order they are consumed; the warp that is last out of a
-  //      slot requests the item kLStages further on into it
-  auto cursor_advance = [&](LaneCursor& c) {
+  // ---- the rings: a warp's items (the phases of its rows) in the order it consumes them; lane 0
+  //      requests item n + kLStages into the slot of item n as soon as the warp has read it
+  // row indices of a parent's rows, for the warps' requests (one thread; slot = parity of the parent)
+  auto fill_rows = [&](int parent) {
+    const int hw = P.h * P.w;
+    const int b = parent / hw, rem = parent - b * hw, ca = rem / P.w, cc = rem - ca * P.w;
+    int* rows = sm.rows[parent & 1];
+    sm.image[parent & 1] = b;
+    rows[0] = parent;
+    int j = 1;
+    for (int di = 0; di < P.r; ++di)
+      for (int dj = 0; dj < P.r; ++dj, ++j) rows[j] = b * N + (ca * P.r + di) * P.W + cc * P.r + dj;
+  };
+  auto cursor_issue = [&](LaneCursor& c, int slot) {   // lane 0 of a warp; steps the cursor
+    const uint32_t dst = wring + (uint32_t)slot * kLSlot;
+    uint64_t* bar = &sm.full[warp][slot];
+    const int row = sm.rows[c.parent & 1][c.j];
+    if (c.j == 0) {
+      mbar_expect_tx(bar, kLTile);
+      tma_tile_3d(dst, &tm_q, IDS * c.ph, 32 * warp, row, bar);
+    } else {
+      mbar_expect_tx(bar, HAS_U ? kLSlot : kLTile);
+      tma_tile_3d(dst, &tm_c, IDS * c.ph, 32 * warp, row, bar);
+      if (HAS_U) tma_tile_3d(dst + kLTile, &tm_u, IDS * c.ph, 32 * warp, row, bar);
+    }
     if (++c.ph == n_ph) {
       c.ph = 0;
       if (++c.j == rows_per_parent) {
         c.j = 0;
         ++c.parent;
-        if (++c.cc == P.w) {
-          c.cc = 0;
-          if (++c.ca == P.h) {
-            c.ca = 0;
-            ++c.b;
-          }
-        }
       }
     }
   };
-  auto cursor_issue = [&](const LaneCursor& c, int slot) {
-    const uint32_t dst = ring + (uint32_t)slot * kLSlot;
-    if (c.j == 0) {
-      mbar_expect_tx(&sm.full[slot], kLTile);
-      tma_tile_3d(dst, &tm_q, IDS * c.ph, 0, c.parent, &sm.full[slot]);
-    } else {
-      const int child = c.j - 1;
-      const int row = c.b * N + (c.ca * P.r + child / P.r) * P.W + c.cc * P.r + child % P.r;
-      mbar_expect_tx(&sm.full[slot], HAS_U ? kLSlot : kLTile);
-      tma_tile_3d(dst, &tm_c, IDS * c.ph, 0, row, &sm.full[slot]);
-      if (HAS_U) tma_tile_3d(dst + kLTile, &tm_u, IDS * c.ph, 0, row, &sm.full[slot]);
-    }
-  };
   if (tid == 0) {
+    fill_rows(p_begin);
+    if (p_begin + 1 < p_end) fill_rows(p_begin + 1);
+  }
+  __syncthreads();
+  if (lane == 0) {
     const int total = (p_end - p_begin) * rows_per_parent * n_ph;
-    const int hw = P.h * P.w;
     LaneCursor cur;
-    cur.ph = 0; cur.j = 0; cur.parent = p_begin; cur.left = 0;
-    cur.b = p_begin / hw; cur.ca = (p_begin % hw) / P.w; cur.cc = (p_begin % hw) % P.w;
-    for (int s = 0; s < kLStages; ++s) {
+    cur.ph = 0; cur.j = 0; cur.parent = p_begin;
+    for (int s = 0; s < kLStages; ++s)
       if (s < total) cursor_issue(cur, s);
-      LaneCursor nxt = cur;
-      for (int k = 0; k < kLStages; ++k) cursor_advance(nxt);
-      nxt.left = total > s + kLStages ? (total - s - 1) / kLStages : 0;
-      sm.cursor[s] = nxt;
-      cursor_advance(cur);
-    }
+    cur.left = total > kLStages ? total - kLStages : 0;
+    sm.cursor[warp] = cur;
   }
   int rs = 0;   // slots consumed so far: bit 0 = the slot to read next, bit 1 = its phase
 #define rslot (rs & 1)
 #define rphase ((uint32_t)(rs >> 1) & 1u)
   static_assert(kLStages == 2, "the packed ring state assumes two slots");
-  auto release_slot = [&]() {
-    __syncwarp();
+  // The warp has the slot's words in registers: request the next item into it.  (`loaded` is one
+  // of those words: naming it here makes the request wait for the warp's shared loads, which are
+  // one instruction for all lanes; the copy's first write then comes hundreds of cycles later.)
+  auto release_slot = [&](uint32_t loaded) {
+    asm volatile("" ::"r"(loaded) : "memory");
     if (lane == 0) {
-      __threadfence_block();
-      const unsigned old = atomicAdd(&sm.done[rslot], 1u);
-      if (old == (unsigned)kLWarps - 1u) {
-        sm.done[rslot] = 0;
-        __threadfence_block();
-        LaneCursor cur = sm.cursor[rslot];
-        if (cur.left > 0) {
-          cursor_issue(cur, rslot);
-          --cur.left;
-#pragma unroll
-          for (int k = 0; k < kLStages; ++k) cursor_advance(cur);
-          sm.cursor[rslot] = cur;
-        }
+      LaneCursor cur = sm.cursor[warp];
+      if (cur.left > 0) {
+        cursor_issue(cur, rslot);
+        --cur.left;
+        sm.cursor[warp] = cur;
       }
     }
     ++rs;
   };
   auto skip_row = [&]() {
     for (int ph = 0; ph < n_ph; ++ph) {
-      lane_wait(&sm.full[rslot], rphase, a.dev_status);
-      release_slot();
+      lane_wait(&sm.full[warp][rslot], rphase, a.dev_status);
+      release_slot(0u);
     }
   };
 
   // ---- pivot, histogram scale and exp reference of the next row of a kind
-  auto choose_pivot = [&](int kind, auto row_u_tag, float& pivot, float& inv_w, float& ref) {
-    constexpr bool ROW_U = decltype(row_u_tag)::value;
-    const LanePredictor pr = sm.pred[kind];
-    if (pr.have) {   // block-uniform
-      pivot = pr.pivot;
-      inv_w = pr.inv_w;
-      ref = pr.ref;
+  auto choose_pivot = [&](int kind, const bool row_u, float& pivot, float& inv_w, float& ref) {
+    if (sm.pred[kind].have) {   // block-uniform
+      pivot = sm.pred[kind].pivot;
+      inv_w = sm.pred[kind].inv_w;
+      ref = sm.pred[kind].ref;
       return;
     }
+    const LanePredictor pr = sm.pred[kind];
     // no prediction: mean and spread of the row's first phase (every thread's first ids: an
     // even sample of the row), assuming a normal shape; the slot is read again by the dense pass
-    lane_wait(&sm.full[rslot], rphase, a.dev_status);
-    const uint32_t sb = ring + (uint32_t)rslot * kLSlot + my_off;
+    lane_wait(&sm.full[warp][rslot], rphase, a.dev_status);
+    const uint32_t sb = wring + (uint32_t)rslot * kLSlot + my_off;
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
       const uint4 c = lds128(sb + (((uint32_t)i ^ sw) << 4));
       uint4 u = make_uint4(0, 0, 0, 0);
-      if (ROW_U) u = lds128(sb + kLTile + (((uint32_t)i ^ sw) << 4));
+      if (row_u) u = lds128(sb + kLTile + (((uint32_t)i ^ sw) << 4));
       const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, uw[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         if (BF16) {
-          const float z0 = mix_logit(bf16_lo(cw[j]), bf16_lo(uw[j]), ROW_U, P.cfg_scale, P.invT);
-          const float z1 = mix_logit(bf16_hi(cw[j]), bf16_hi(uw[j]), ROW_U, P.cfg_scale, P.invT);
+          const float z0 = mix_logit(bf16_lo(cw[j]), bf16_lo(uw[j]), row_u, P.cfg_scale, P.invT);
+          const float z1 = mix_logit(bf16_hi(cw[j]), bf16_hi(uw[j]), row_u, P.cfg_scale, P.invT);
           s1 += z0 + z1;
           s2 += z0 * z0 + z1 * z1;
         } else {
-          const float z0 = mix_logit(__uint_as_float(cw[j]), __uint_as_float(uw[j]), ROW_U, P.cfg_scale, P.invT);
+          const float z0 = mix_logit(__uint_as_float(cw[j]), __uint_as_float(uw[j]), row_u, P.cfg_scale, P.invT);
           s1 += z0;
           s2 += z0 * z0;
         }
@@ -453,56 +522,79 @@ __global__ void __launch_bounds__(kLThreads, 3)
     const float sd = sqrtf(fmaxf((float)(S2 / cnt) - mean * mean, 1e-20f));
     const float d = fmaxf((a.a_theta - a.a_boot) * sd, 1e-20f);
     pivot = mean + (a.a_boot + pr.shift) * sd;
-    inv_w = (float)kLBins / (3.0f * d);
+    inv_w = (float)kLBins / (2.0f * d);
     ref = mean + a.a_max * sd;
   };
 
-  // ---- a row through the ring into this thread's list; returns the entry count
-  auto stream_row = [&](auto row_u_tag, uint32_t base, uint32_t lim, float pivot, uint32_t& m_lo, uint32_t& m_hi) -> int {
-    constexpr bool ROW_U = decltype(row_u_tag)::value;
+  // ---- a row through the ring into this thread's list (from `base` towards `lim`, the first row of
+  //      the stack it grows towards); returns the entry count.  Before a phase the thread makes sure
+  //      that a whole phase's worth of rows is left; if not, its cursor stops (the appends of the
+  //      rest of the row land on one row) and the row is given up after the next barrier.
+  auto stream_row = [&](LaneSel& sel, const bool row_u, uint32_t base, uint32_t lim, float pivot, uint32_t& m_lo,
+                        uint32_t& m_hi) -> int {
     uint32_t cur = base;
     m_lo = 0;
     m_hi = 0;
 #pragma unroll 1
     for (int ph = 0; ph < n_ph; ++ph) {
-      lane_wait(&sm.full[rslot], rphase, a.dev_status);
-      const uint32_t sb = ring + (uint32_t)rslot * kLSlot + my_off;
-      uint32_t m;
-      // the four variants differ in compile-time constants only; the branch is warp-uniform
-      if (up) {
-        m = scale ? lane_dense<BF16, ROW_U, true, 512>(sb, sw, P.cfg_scale, P.invT, pivot, cur, lim)
-                  : lane_dense<BF16, ROW_U, false, 512>(sb, sw, P.cfg_scale, P.invT, pivot, cur, lim);
-      } else {
-        m = scale ? lane_dense<BF16, ROW_U, true, -512>(sb, sw, P.cfg_scale, P.invT, pivot, cur, lim)
-                  : lane_dense<BF16, ROW_U, false, -512>(sb, sw, P.cfg_scale, P.invT, pivot, cur, lim);
+      lane_wait(&sm.full[warp][rslot], rphase, a.dev_status);
+      const uint32_t room = (up ? lim - cur : cur - lim) >> 9;   // rows between the cursor and the other stack
+      uint32_t stp = (uint32_t)step;
+      if (room < (uint32_t)IDS) {
+        stp = 0u;
+        sel.overflow = 1;
       }
-      release_slot();
+      uint4 c[2], u[2];
+      uint32_t m;
+      const uint32_t sb = wring + (uint32_t)rslot * kLSlot + my_off;
+      // (the variants differ in compile-time constants only; the branches are block-uniform)
+      if (HAS_U && row_u) {
+        lane_load<true>(sb, sw, c, u);
+        release_slot(c[1].w ^ u[1].w);
+        m = scale ? lane_dense<BF16, true, true>(c, u, P.cfg_scale, P.invT, pivot, cur, stp)
+                  : lane_dense<BF16, true, false>(c, u, P.cfg_scale, P.invT, pivot, cur, stp);
+      } else {
+        lane_load<false>(sb, sw, c, u);
+        release_slot(c[1].w);
+        m = scale ? lane_dense<BF16, false, true>(c, u, P.cfg_scale, P.invT, pivot, cur, stp)
+                  : lane_dense<BF16, false, false>(c, u, P.cfg_scale, P.invT, pivot, cur, stp);
+      }
       const int bit0 = ph * IDS;
       if (bit0 < 32) m_lo |= m << bit0;
       else m_hi |= m << (bit0 - 32);
     }
-    return up ? (int)((cur - base) >> 9) : (int)((base - cur) >> 9);
+    return (int)((up ? cur - base : base - cur) >> 9);
   };
 
   // ---- pass 1 over the thread's own entries: exp against the reference, maximum, histogram of
   //      the low end; per-warp partial results for the block
-  auto pass_one = [&](LaneSel& sel, uint32_t base, int n, float pivot, float inv_w, float c0, uint32_t& lowm) {
+  auto pass_one = [&](LaneSel& sel, uint32_t base, int n, float pivot, float inv_w, float c0, uint32_t& lowm) -> float {
     const float hoff = -pivot * inv_w;
     float mx = -INFINITY, s_all = 0.f;
     lowm = 0;
+    // four entries per trip, every warp lane making the same number of trips (a lane past its own
+    // end loads nothing and works on -inf: no weight, no bin), so that the four chains of
+    // load -> exp -> add overlap and the loop needs no divergence handling
+    const int nmax = __reduce_max_sync(kFull, n);
     uint32_t ad = base;
-#pragma unroll 2
-    for (int i = 0; i < n; ++i, ad += step) {
-      const float z = lds_f32(ad);
-      mx = fmaxf(mx, z);
-      s_all += ex2f(fmaf(z, kLog2e, c0));
-      // (a column whose stacks have met holds entries from below the pivot until the row is
-      // given up after the next barrier: the unsigned compare keeps their bins out of range)
-      const unsigned bin = (unsigned)(int)fmaf(z, inv_w, hoff);
-      if (bin < (unsigned)kLBins) {
-        atomicAdd(&sel.hist[bin], 1u);
-        lowm |= 1u << (i & 31);
+    for (int i0 = 0; i0 < nmax; i0 += 4, ad += 4 * step) {
+      float z[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) z[k] = i0 + k < n ? lds_f32(ad + (uint32_t)(k * step)) : -INFINITY;
+      uint32_t low4 = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        mx = fmaxf(mx, z[k]);
+        s_all += ex2f(fmaf(z[k], kLog2e, c0));
+        // (a column whose stacks have met holds entries from below the pivot until the row is
+        // given up after the next barrier: the unsigned compare keeps their bins out of range)
+        const unsigned bin = (unsigned)(int)fmaf(z[k], inv_w, hoff);
+        if (bin < (unsigned)kLBins) {
+          atomicAdd(&sel.hist[bin], 1u);
+          low4 |= 1u << k;
+        }
       }
+      lowm |= low4 << (i0 & 31);
     }
     sm.cnt[tid] = (unsigned char)n;
     const int nsum = __reduce_add_sync(kFull, n);
@@ -513,6 +605,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
       sel.w_max[warp] = key_float(mk);
       sel.w_e[warp] = es;
     }
+    return s_all;   // exp of ALL of this thread's entries, in list order
   };
 
   struct Sel {
@@ -531,10 +624,10 @@ __global__ void __launch_bounds__(kLThreads, 3)
     s.n = n;
     s.mx = mx;
     s.reason = 0;
-    // the two stacks that grow towards each other must not (nearly) fill the `rows` they share;
-    // the bit mask of a thread's low entries covers 32 entries
+    // the two stacks that grow towards each other must fit the `rows` they share; the bit mask of a
+    // thread's low entries covers 32 entries
     const int mine_n = sm.cnt[tid], other_n = sm.cnt[tid ^ 128];
-    if (__any_sync(kFull, mine_n + other_n >= rows - 1 || mine_n > 32) && lane == 0) sel.overflow = 1;
+    if (__any_sync(kFull, mine_n + other_n > rows || mine_n > 32) && lane == 0) sel.overflow = 1;
     if (n < P.top_k) {
       s.reason = 2;
       return false;
@@ -545,13 +638,17 @@ __global__ void __launch_bounds__(kLThreads, 3)
     }
     const int rank = n - P.top_k + 1;   // 1-based rank from the bottom of the k-th largest
     constexpr int PER = kLBins / 32;
+    static_assert(PER == 8, "a lane reads its eight bins with two 128-bit loads");
     unsigned h[PER];
+    {
+      const uint4 h0 = *reinterpret_cast<const uint4*>(&sel.hist[lane * PER]);
+      const uint4 h1 = *reinterpret_cast<const uint4*>(&sel.hist[lane * PER + 4]);
+      h[0] = h0.x; h[1] = h0.y; h[2] = h0.z; h[3] = h0.w;
+      h[4] = h1.x; h[5] = h1.y; h[6] = h1.z; h[7] = h1.w;
+    }
     unsigned mine = 0;
 #pragma unroll
-    for (int b = 0; b < PER; ++b) {
-      h[b] = sel.hist[lane * PER + b];
-      mine += h[b];
-    }
+    for (int b = 0; b < PER; ++b) mine += h[b];
     unsigned inc = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -590,26 +687,39 @@ __global__ void __launch_bounds__(kLThreads, 3)
 
   // between the first and the second barrier: the thread's low entries once more -- those below the
   // crossing bin leave the partition sum, those inside it are set aside to be ranked exactly
-  auto set_aside = [&](LaneSel& sel, uint32_t base, uint32_t lowm, float pivot, float inv_w, float c0, int bstar) {
+  auto set_aside = [&](LaneSel& sel, uint32_t base, uint32_t lowm, float pivot, float inv_w, float c0, int bstar) -> float {
     const float hoff = -pivot * inv_w;
     float excl = 0.f;
-    while (lowm) {
-      const int i = __ffs(lowm) - 1;
-      lowm &= lowm - 1;
-      const float z = lds_f32(base + (uint32_t)(i * step));
-      const int bin = (int)fmaf(z, inv_w, hoff);
-      const float e = ex2f(fmaf(z, kLog2e, c0));
-      if (bin < bstar) excl += e;
-      else if (bin == bstar) {
-        const unsigned at = atomicAdd(&sel.n_sa, 1u);
-        if (at < (unsigned)kLSetAside) {
-          sel.sa_z[at] = z;
-          sel.sa_e[at] = e;
-        }
+    // four low entries per trip (their loads and bins overlap); a thread has two or three on average
+    const int trips = (__reduce_max_sync(kFull, __popc(lowm)) + 3) >> 2;
+    for (int it = 0; it < trips; ++it) {
+      float z[4];
+      int bin[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = __ffs(lowm) - 1;   // -1: none left
+        lowm &= lowm - 1;
+        z[k] = i >= 0 ? lds_f32(base + (uint32_t)(i * step)) : INFINITY;
+        bin[k] = (int)fmaf(z[k], inv_w, hoff);   // +inf -> a bin above every other
       }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (bin[k] <= bstar) {
+          const float e = ex2f(fmaf(z[k], kLog2e, c0));
+          if (bin[k] < bstar) excl += e;
+          else {
+            const unsigned at = atomicAdd(&sel.n_sa, 1u);
+            if (at < (unsigned)kLSetAside) {
+              sel.sa_z[at] = z[k];
+              sel.sa_e[at] = e;
+              sel.sa_owner[at] = (unsigned short)tid;
+            }
+          }
+        }
     }
     const double ex = warp_sum((double)excl);
     if (lane == 0) sel.w_excl[warp] = ex;
+    return excl;   // exp of this thread's entries below the crossing bin
   };
 
   // after the second barrier: the exact k-th largest value, the number of entries >= it and the
@@ -653,45 +763,6 @@ __global__ void __launch_bounds__(kLThreads, 3)
     return true;
   };
 
-  auto learn = [&](int kind, bool ok, int reason, float theta, float pivot, int n, int n_ge, float mx) {
-    LanePredictor pr = sm.pred[kind];
-    if (!ok) {
-      pr.have = 0;
-      const int dir = reason == 2 ? -1 : (reason == 1 || reason == 3) ? 1 : 0;
-      if (dir != 0) {
-        const float unit = 0.5f * (a.a_theta - a.a_boot);
-        if (pr.dir == 0) pr.step = unit;
-        else if (pr.dir == dir) pr.step = fminf(2.0f * pr.step, 64.0f * unit);
-        else pr.step = fmaxf(0.5f * pr.step, 0.25f * unit);
-        pr.shift += (float)dir * pr.step;
-        pr.dir = dir;
-      }
-    } else {
-      pr.dir = 0;
-      const int below = n - n_ge;   // candidates in [pivot, theta)
-      float rho = pr.rho;
-      bool rho_ok = pr.have != 0;
-      if (theta > pivot && below >= 16) {
-        const float r_new = (float)below / (theta - pivot);
-        rho = pr.have ? pr.rho + 0.25f * (r_new - pr.rho) : r_new;
-        rho_ok = true;
-      }
-      if (!rho_ok) {
-        pr.have = 0;
-      } else {
-        pr.theta = pr.have ? pr.theta + 0.25f * (theta - pr.theta) : theta;
-        pr.mx = pr.have ? pr.mx + 0.25f * (mx - pr.mx) : mx;
-        pr.rho = rho;
-        pr.have = 1;
-        const float d = (float)a.margin / rho;
-        pr.pivot = pr.theta - d;
-        pr.inv_w = (float)kLBins / (3.0f * d);
-        pr.ref = pr.mx;
-      }
-    }
-    sm.pred[kind] = pr;
-  };
-
   auto count_failure = [&](int reason) {   // one thread
     if (reason < 1 || reason > 4) return;
     const int slot = reason == 1 ? kCntListFull : reason == 2 ? kCntTooFew : reason == 3 ? kCntAboveRange : kCntCrowdedBin;
@@ -719,182 +790,244 @@ __global__ void __launch_bounds__(kLThreads, 3)
 
   if (tid == kLThreads - 1) sm.tok[p_begin & 1] = __ldg(a.draft_tok_lo + p_begin);
   for (int parent = p_begin; parent < p_end; ++parent) {
-    // position of the parent's first child: image pb, raster index t0 within the image
-    int pb, t0;
-    {
-      const int hw = P.h * P.w;
-      pb = parent / hw;
-      const int rem = parent - pb * hw, pca = rem / P.w, pcc = rem - pca * P.w;
-      t0 = pca * P.r * P.W + pcc * P.r;
-    }
-    bool q_ok;
-    // ------------------------------------------------------------ draft row
-    {
+    const int pb = sm.image[parent & 1];   // (tables written at least two barriers ago)
+    // One loop body for the draft row (j = 0) and the r*r target rows under it: the two kinds of row
+    // share every pass up to the exact threshold, and one copy of the code is what the
+    // instruction cache holds.
+#pragma unroll 1
+    for (int j = 0; j <= rr; ++j) {
+      const bool is_q = j == 0;
       LaneSel& sel = sm.sel[rowi & 1];
+      LanePrep& pp = sm.prep[rowi & 1];
       ++rowi;
+      const size_t g = (size_t)sm.rows[parent & 1][j];   // a target row's position b * N + t (the draft row's cell)
+      const int t = (int)g - pb * N;
       float pivot, inv_w, ref;
-      choose_pivot(0, std::false_type{}, pivot, inv_w, ref);
+      choose_pivot(is_q ? 0 : 1, HAS_U && !is_q, pivot, inv_w, ref);
       const float c0 = -ref * kLog2e;
+      // Two threads prepare what the row needs besides its lists: the logit of x~ (requested here by
+      // asynchronous copies, read after the row has been streamed, so that no warp sits on the load)
+      // and the position's uniforms.
       if (tid == kLThreads - 1) {
-        // the draft logit of x~ and the next parent's token: requested now, read after the row
-        cp_async_wait_all();
-        const int tok = checked_token(sm.tok[parent & 1], P.V, a.dev_status);
-        sm.tok[parent & 1] = tok;
-        cp_async4(&sm.raw_q, logit_word<BF16>(a.draft, (size_t)parent * P.V + (size_t)tok));
-        if (parent + 1 < p_end) cp_async4(&sm.tok[(parent + 1) & 1], a.draft_tok_lo + parent + 1);
+        if (is_q) {
+          cp_async_wait_all();   // the token, requested a parent ago
+          const int tok = checked_token(sm.tok[parent & 1], P.V, a.dev_status);
+          sm.tok[parent & 1] = tok;
+          cp_async4(&sm.raw_q, logit_word<BF16>(a.draft, (size_t)parent * P.V + (size_t)tok));
+          if (parent + 1 < p_end) cp_async4(&sm.tok[(parent + 1) & 1], a.draft_tok_lo + parent + 1);
+        } else {
+          const size_t at = g * (size_t)P.V + (size_t)sm.tok[parent & 1];
+          cp_async4(&pp.raw_c, logit_word<BF16>(a.cond, at));
+          if (HAS_U) cp_async4(&pp.raw_u, logit_word<BF16>(a.uncond, at));
+        }
+      } else if (tid == kLThreads - 33 && !is_q) {
+        const uint4 rnd = lane_philox(make_uint4((uint32_t)t, (uint32_t)pb + P.image_offset, P.round, 0u),
+                                      make_uint2(P.seed_lo, P.seed_hi));
+        pp.rnd[0] = rnd.x;
+        pp.rnd[1] = rnd.y;
+        pp.rnd[2] = rnd.z;
       }
-      nq = stream_row(std::false_type{}, q_base, q_lim, pivot, dm_lo, dm_hi);
+      // where the row's entries go: the draft row's from the end of the column, a target row's from
+      // the end of the thread's draft entries, up to the first target row of the other thread
+      const uint32_t base = is_q ? q_base : q_base + (uint32_t)(nq * step);
+      const uint32_t lim = is_q ? q_lim : q_lim - (uint32_t)(nq_other * step);
+      uint32_t m_lo, m_hi;
+      const int n = stream_row(sel, HAS_U && !is_q, base, lim, pivot, m_lo, m_hi);
       uint32_t lowm;
-      pass_one(sel, q_base, nq, pivot, inv_w, c0, lowm);
+      const float s_all = pass_one(sel, base, n, pivot, inv_w, c0, lowm);
+      if (tid == kLThreads - 1 && !is_q) {
+        cp_async_wait_all();
+        const size_t at = g * (size_t)P.V + (size_t)sm.tok[parent & 1];
+        const float z = mix_logit(logit_of_word<BF16>(pp.raw_c, at), HAS_U ? logit_of_word<BF16>(pp.raw_u, at) : 0.f,
+                                  HAS_U, P.cfg_scale, P.invT);
+        pp.z_tok = z;
+        pp.e_tok = lane_exp2((double)z * (double)kLog2e + (double)c0);   // the list entries' own exponent
+      }
       __syncthreads();   // ---- barrier 1
       reset_selection(sm.sel[rowi & 1]);
       Sel s;
-      bool ok = locate_bin(sel, s, ref, R);
-      nq_other = sm.cnt[tid ^ 128];
-      if (ok) set_aside(sel, q_base, lowm, pivot, inv_w, c0, s.bstar);
+      bool ok = locate_bin(sel, s, ref, is_q ? R : R - nq - nq_other);
+      if (is_q) {
+        nq_other = sm.cnt[tid ^ 128];
+        // the warps are requesting rows of this parent and (at its end) of the next; the table entry of
+        // the parent after that replaces the previous parent's, whose last request is behind every warp
+        if (tid == 64 && parent + 1 < p_end && parent > p_begin) fill_rows(parent + 1);
+      }
+      float s_inc = s_all;   // becomes: exp of this thread's entries that are >= theta
+      if (ok) s_inc -= set_aside(sel, base, lowm, pivot, inv_w, c0, s.bstar);
       __syncthreads();   // ---- barrier 2
       float theta = 0.f;
       int n_ge = 0;
-      double Zq = 1.0;
+      double Z = 1.0;
       if (ok && sel.overflow) {
         ok = false;
         s.reason = 1;
       }
-      if (ok) ok = finish_selection(sel, s, theta, n_ge, Zq);
-      if (ok && !(Zq > 0.0 && Zq < 1e300)) ok = false;
-      if (ok) {
-        // q in place of z: q(x) = [z >= theta] exp(z - ref) / Z_q, the fp32 product of e and 1/Z_q
-        const float invZq = (float)(1.0 / Zq);
-        uint32_t ad = q_base;
-#pragma unroll 2
-        for (int i = 0; i < nq; ++i, ad += step) {
-          const float z = lds_f32(ad);
-          const float e = ex2f(fmaf(z, kLog2e, c0));
-          sts_f32(ad, z >= theta ? __fmul_rn(e, invZq) : 0.f);
+      if (ok) ok = finish_selection(sel, s, theta, n_ge, Z);
+      if (ok && !(Z > 0.0 && Z < 1e300)) ok = false;
+      if (tid == kLThreads - 1)
+        lane_learn(&sm.pred[is_q ? 0 : 1], ok, s.reason, theta, pivot, s.n, n_ge, s.mx, a.margin, a.a_theta, a.a_boot);
+
+      if (is_q) {
+        // ------------------------------------------------------------ the draft row ends here
+        if (!ok) {   // block-uniform: the whole parent goes to the general routines
+          if (tid == 0) {
+            atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
+            count_failure(s.reason);
+            for (int ch = 1; ch <= rr; ++ch) defer((size_t)sm.rows[parent & 1][ch]);
+          }
+          for (int ch = 0; ch < rr; ++ch) skip_row();
+          __syncthreads();   // the predictor written above is read by the next draft row
+          break;
         }
-      }
-      if (tid == kLThreads - 1) {
-        if (ok) {
+        dm_lo = m_lo;
+        dm_hi = m_hi;
+        nq = n;
+        {   // q in place of z: q(x) = [z >= theta] exp(z - ref) / Z_q, the fp32 product of e and 1/Z_q
+          const float invZq = 1.0f / (float)Z;
+          uint32_t ad = q_base;
+#pragma unroll 2
+          for (int i = 0; i < nq; ++i, ad += step) {
+            const float z = lds_f32(ad);
+            const float e = ex2f(fmaf(z, kLog2e, c0));
+            sts_f32(ad, z >= theta ? __fmul_rn(e, invZq) : 0.f);
+          }
+        }
+        if (tid == kLThreads - 1) {
           cp_async_wait_all();
           const size_t at = (size_t)parent * P.V + (size_t)sm.tok[parent & 1];
           const float zq_tok = mix_logit(logit_of_word<BF16>(sm.raw_q, at), 0.f, false, 0.f, P.invT);
           // the same exponent as the list entries: 2^(z * fp32(log2 e) + c0)
-          const double q = (zq_tok >= theta) ? exp2((double)zq_tok * (double)kLog2e + (double)c0) / Zq : 0.0;
+          const double q = (zq_tok >= theta) ? lane_exp2((double)zq_tok * (double)kLog2e + (double)c0) / Z : 0.0;
           if (q <= 0.0) atomicOr(a.dev_status, MULO_DEV_ZERO_DRAFT_PROB);
           sm.q_tok = q;
-        } else {
+        }
+        continue;
+      }
+
+      // ------------------------------------------------------------ a target row goes on
+      if (!ok) {   // block-uniform
+        if (tid == 0) {
           atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
           count_failure(s.reason);
-          for (int child = 0; child < rr; ++child)
-            defer((size_t)pb * N + t0 + (child / P.r) * P.W + child % P.r);
+          defer(g);
         }
-        learn(0, ok, s.reason, theta, pivot, s.n, n_ge, s.mx);
+        __syncthreads();   // the predictor
+        continue;
       }
-      q_ok = ok;
-    }
+      {   // this thread's entries of the crossing bin that fell below theta
+        const int mcount = (int)sel.n_sa;
+        for (int i = 0; i < mcount; ++i)
+          if (sel.sa_owner[i] == tid && sel.sa_z[i] < theta) s_inc -= sel.sa_e[i];
+        s_inc = fmaxf(s_inc, 0.f);
+      }
+      // ---- the decision (Eq. 1 / Eq. 5), the same in every thread
+      const double e_tok = (pp.z_tok >= theta) ? pp.e_tok : 0.0;
+      const double q_tok = sm.q_tok;
+      int accepted;
+      if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = e_tok >= P.tau * Z;
+      else if (q_tok <= 0.0) accepted = e_tok > 0.0;
+      else accepted = uniform24(pp.rnd[0]) * q_tok * Z < e_tok;
+      const float invZp = 1.0f / (float)Z;
+      if (tid == 0) {
+        a.flags[g] = accepted ? 0 : 1;
+        if (a.p_tok || a.q_tok || a.accept_prob)
+          lane_write_probs(a.p_tok, a.q_tok, a.accept_prob, g, e_tok, q_tok, Z, P.accept_mode == MULO_ACCEPT_THRESHOLD);
+      }
 
-    // ------------------------------------------------------------ children
-    if (!q_ok) {   // block-uniform: the whole parent went to the general routines
-      for (int child = 0; child < rr; ++child) skip_row();
-      __syncthreads();   // the predictor written above is read by the next draft row
-    } else {
-      // where this thread's target entries go: above (below) its own draft entries, up to the first
-      // target row of the thread it shares the column with
-      const uint32_t t_base = q_base + (uint32_t)(nq * step);
-      const uint32_t t_lim = q_lim - (uint32_t)(nq_other * step);
-      for (int child = 0; child < rr; ++child) {
-        LaneSel& sel = sm.sel[rowi & 1];
-        LanePrep& pp = sm.prep[rowi & 1];
-        ++rowi;
-        const int t = t0 + (child / P.r) * P.W + child % P.r;
-        const size_t g = (size_t)pb * N + t;
-        float pivot, inv_w, ref;
-        choose_pivot(1, std::integral_constant<bool, HAS_U>{}, pivot, inv_w, ref);
-        const float c0 = -ref * kLog2e;
-        // Two threads prepare the position's uniforms and exp of the logit of x~ (in double).  The
-        // logit's words are requested here by asynchronous copies and read after the row has been
-        // streamed, so that no warp sits on the load.
-        if (tid == kLThreads - 1) {
-          const size_t at = g * (size_t)P.V + (size_t)sm.tok[parent & 1];
-          cp_async4(&pp.raw_c, logit_word<BF16>(a.cond, at));
-          if (HAS_U) cp_async4(&pp.raw_u, logit_word<BF16>(a.uncond, at));
-        } else if (tid == kLThreads - 33) {
-          const uint4 rnd = philox4x32_10(make_uint4((uint32_t)t, (uint32_t)pb + P.image_offset, P.round, 0u),
-                                          make_uint2(P.seed_lo, P.seed_hi));
-          pp.rnd[0] = rnd.x;
-          pp.rnd[1] = rnd.y;
-          pp.rnd[2] = rnd.z;
-        }
-        uint32_t m_lo, m_hi;
-        const int n = stream_row(std::integral_constant<bool, HAS_U>{}, t_base, t_lim, pivot, m_lo, m_hi);
-        uint32_t lowm;
-        pass_one(sel, t_base, n, pivot, inv_w, c0, lowm);
-        if (tid == kLThreads - 1) {
-          cp_async_wait_all();
-          const size_t at = g * (size_t)P.V + (size_t)sm.tok[parent & 1];
-          const float z = mix_logit(logit_of_word<BF16>(pp.raw_c, at), HAS_U ? logit_of_word<BF16>(pp.raw_u, at) : 0.f,
-                                    HAS_U, P.cfg_scale, P.invT);
-          pp.z_tok = z;
-          pp.e_tok = exp2((double)z * (double)kLog2e + (double)c0);   // the list entries' own exponent
-        }
-        __syncthreads();   // ---- barrier 1
-        reset_selection(sm.sel[rowi & 1]);
-        Sel s;
-        bool ok = locate_bin(sel, s, ref, R - nq - nq_other);
-        if (ok) set_aside(sel, t_base, lowm, pivot, inv_w, c0, s.bstar);
-        __syncthreads();   // ---- barrier 2
-        float theta = 0.f;
-        int n_ge = 0;
-        double Zp = 1.0;
-        if (ok && sel.overflow) {
-          ok = false;
-          s.reason = 1;
-        }
-        if (ok) ok = finish_selection(sel, s, theta, n_ge, Zp);
-        if (ok && !(Zp > 0.0 && Zp < 1e300)) ok = false;
-        if (tid == kLThreads - 1) learn(1, ok, s.reason, theta, pivot, s.n, n_ge, s.mx);
-        if (!ok) {   // block-uniform
-          if (tid == 0) {
-            atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
-            count_failure(s.reason);
-            defer(g);
+      // ---- the draws (one copy of the code: a loop over the draws the position needs).
+      // A draw = the thread's sum, a block scan in double, ONE barrier, and the walk of the thread
+      // that owns u * total.  Weight of an entry: residual max(0, e / Z_p - q) with q from the draft
+      // row's list of this thread (found by popcount on the two masks), or target e; entries below
+      // theta weigh nothing.  A residual without mass is drawn again from the target weights with
+      // the same uniform.
+      const uint32_t t_base = base;
+      const int n_lo = __popc(m_lo), nq_lo = __popc(dm_lo);
+      int pending = draws_for(P.resample_mode, accepted);   // bit 0 residual, bit 1 target
+      bool no_mass = false;
+      int dcall = 0;   // consecutive draws alternate between the two scan buffers
+#pragma unroll 1
+      while (pending) {
+        const bool is_res = (pending & kDrawResidual) != 0;
+        const bool resid = is_res && !no_mass;
+        const double u = uniform24(pp.rnd[is_res ? 1 : 2]);
+        int32_t* const out = (is_res ? a.cand_res : a.cand_tgt) + g;
+        // The thread's sum needs no pass over its list.  Target weights: the exps of its entries
+        // >= theta are known already (s_inc).  Residual: max(0, p - q) = p - min(p, q), and
+        // min(p, q) is not zero only for ids that BOTH rows kept, so the sum is s_inc / Z_p minus
+        // the min over the intersection of the two masks (about a third of the entries).
+        float S = s_inc;
+        if (resid) {
+          auto both = [&](uint32_t bit, uint32_t m, uint32_t dm, uint32_t tb, uint32_t qb) -> float {
+            const uint32_t below = bit - 1u;
+            const float z = bit ? lds_f32(tb + (uint32_t)(__popc(m & below) * step)) : -INFINITY;
+            const float q = bit ? lds_f32(qb + (uint32_t)(__popc(dm & below) * step)) : 0.f;
+            const float pe = __fmul_rn(ex2f(fmaf(z, kLog2e, c0)), invZp);
+            return z >= theta ? fminf(pe, q) : 0.f;
+          };
+          float mins = 0.f;
+#pragma unroll 1
+          for (int hf = 0; hf < 2; ++hf) {
+            const uint32_t m = hf ? m_hi : m_lo, dm = hf ? dm_hi : dm_lo;
+            const uint32_t tb = hf ? t_base + (uint32_t)(n_lo * step) : t_base;
+            const uint32_t qb = hf ? q_base + (uint32_t)(nq_lo * step) : q_base;
+            uint32_t im = m & dm;
+            const int trips = (__reduce_max_sync(kFull, __popc(im)) + 1) >> 1;
+            for (int it = 0; it < trips; ++it) {   // two entries per trip: their chains overlap
+              const uint32_t b0 = im & (0u - im);
+              im ^= b0;
+              const uint32_t b1 = im & (0u - im);
+              im ^= b1;
+              const float v0 = both(b0, m, dm, tb, qb), v1 = both(b1, m, dm, tb, qb);
+              mins += v0;
+              mins += v1;
+            }
           }
-          __syncthreads();   // the predictor
+          S = fmaxf(__fmul_rn(s_inc, invZp) - mins, 0.f);
+        }
+        // inclusive scan over the warp's threads (ascending ids), warp totals to shared memory
+        double inc = (double)S;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const double v = __shfl_up_sync(kFull, inc, o);
+          if (lane >= o) inc += v;
+        }
+        double excl = __shfl_up_sync(kFull, inc, 1);
+        if (lane == 0) excl = 0.0;
+        double* const wt = sm.w_tot[dcall & 1];
+        ++dcall;
+        if (lane == 31) wt[warp] = inc;
+        __syncthreads();
+        double before = 0.0, total = 0.0;
+#pragma unroll
+        for (int w = 0; w < kLWarps; ++w) {
+          const double v = wt[w];
+          if (w == warp) before = total;
+          total += v;
+        }
+        if (!(total > 0.0)) {   // block-uniform
+          if (resid) {
+            no_mass = true;   // the same draw again, from the target weights
+            continue;
+          }
+          pending &= ~(is_res ? kDrawResidual : kDrawTarget);
+          no_mass = false;
           continue;
         }
-        // ---- the decision (Eq. 1 / Eq. 5), the same in every thread
-        const double e_tok = (pp.z_tok >= theta) ? pp.e_tok : 0.0;
-        const double q_tok = sm.q_tok;
-        int accepted;
-        if (P.accept_mode == MULO_ACCEPT_THRESHOLD) accepted = e_tok >= P.tau * Zp;
-        else if (q_tok <= 0.0) accepted = e_tok > 0.0;
-        else accepted = uniform24(pp.rnd[0]) * q_tok * Zp < e_tok;
-        const int draws = draws_for(P.resample_mode, accepted);
-        const float invZp = (float)(1.0 / Zp);
-        if (tid == 0) {
-          a.flags[g] = accepted ? 0 : 1;
-          if (a.p_tok) a.p_tok[g] = (float)(e_tok / Zp);
-          if (a.q_tok) a.q_tok[g] = (float)q_tok;
-          if (a.accept_prob) {
-            const double p = e_tok / Zp;
-            double thr;
-            if (P.accept_mode == MULO_ACCEPT_THRESHOLD) thr = p;
-            else if (q_tok <= 0.0) thr = p > 0.0 ? 1.0 : 0.0;
-            else thr = fmin(1.0, p / q_tok);
-            a.accept_prob[g] = (float)thr;
-          }
-        }
-
-        // ---- the draws.  Weight of an entry (value z, local id = the next set bit of the mask):
-        //      residual: max(0, e / Z_p - q) with q from the draft row's list of this thread
-        //      (found by popcount on the two masks); target: e.  Entries below theta weigh nothing.
-        // One call = the thread's sum, a block scan in double, ONE barrier, and the walk of the
-        // thread that owns u * total.  Returns false when the weights have no mass.
-        int dcall = 0;   // consecutive draws of a row alternate between the two scan buffers
-        auto draw = [&](bool resid, double u, int32_t* out) -> bool {
-          auto half_sum = [&](uint32_t m, uint32_t dm, uint32_t ad, int qfirst, float acc) -> float {
-            const uint32_t qb = q_base + (uint32_t)(qfirst * step);
-            while (m) {
+        const double y = u * total;
+        const double lo = before + excl, hi = before + inc;
+        if (lo <= y && y < hi) {
+          // this thread owns u * total: walk its entries with the same arithmetic and order
+          int pick = -1, last_pos = -1;
+          float acc = 0.f;
+#pragma unroll 1
+          for (int hf = 0; hf < 2 && pick < 0; ++hf) {
+            uint32_t m = hf ? m_hi : m_lo;
+            const uint32_t dm = hf ? dm_hi : dm_lo;
+            uint32_t ad = hf ? t_base + (uint32_t)(n_lo * step) : t_base;
+            const uint32_t qb = hf ? q_base + (uint32_t)(nq_lo * step) : q_base;
+            const int id0 = tid * W + 32 * hf;
+            while (m && pick < 0) {
               const uint32_t bit = m & (0u - m);
               m ^= bit;
               const float z = lds_f32(ad);
@@ -904,70 +1037,24 @@ __global__ void __launch_bounds__(kLThreads, 3)
                 w = __fmul_rn(w, invZp);
                 if (dm & bit) w = fmaxf(__fsub_rn(w, lds_f32(qb + (uint32_t)(__popc(dm & (bit - 1u)) * step))), 0.f);
               }
-              if (z >= theta) acc += w;
-            }
-            return acc;
-          };
-          const int n_lo = __popc(m_lo), nq_lo = __popc(dm_lo);
-          float S = half_sum(m_lo, dm_lo, t_base, 0, 0.f);
-          S = half_sum(m_hi, dm_hi, t_base + (uint32_t)(n_lo * step), nq_lo, S);
-          // inclusive scan over the warp's threads (ascending ids), warp totals to shared memory
-          double inc = (double)S;
-#pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const double v = __shfl_up_sync(kFull, inc, o);
-            if (lane >= o) inc += v;
-          }
-          double excl = __shfl_up_sync(kFull, inc, 1);
-          if (lane == 0) excl = 0.0;
-          double* const wt = sm.w_tot[dcall & 1];
-          ++dcall;
-          if (lane == 31) wt[warp] = inc;
-          __syncthreads();
-          double before = 0.0, total = 0.0;
-#pragma unroll
-          for (int w = 0; w < kLWarps; ++w) {
-            const double v = wt[w];
-            if (w == warp) before = total;
-            total += v;
-          }
-          if (!(total > 0.0)) return false;
-          const double y = u * total;
-          const double lo = before + excl, hi = before + inc;
-          if (lo <= y && y < hi) {
-            // this thread owns u * total: walk its entries with the same arithmetic and order
-            int pick = -1, last_pos = -1;
-            float acc = 0.f;
-            auto half_walk = [&](uint32_t m, uint32_t dm, uint32_t ad, int qfirst, int id0) {
-              const uint32_t qb = q_base + (uint32_t)(qfirst * step);
-              while (m && pick < 0) {
-                const uint32_t bit = m & (0u - m);
-                m ^= bit;
-                const float z = lds_f32(ad);
-                ad += step;
-                float w = ex2f(fmaf(z, kLog2e, c0));
-                if (resid) {
-                  w = __fmul_rn(w, invZp);
-                  if (dm & bit) w = fmaxf(__fsub_rn(w, lds_f32(qb + (uint32_t)(__popc(dm & (bit - 1u)) * step))), 0.f);
-                }
-                if (z >= theta && w > 0.f) {
-                  acc += w;
-                  last_pos = id0 + __ffs(bit) - 1;
-                  if (lo + (double)acc > y) pick = last_pos;
-                }
+              if (z >= theta && w > 0.f) {
+                acc += w;
+                last_pos = id0 + __ffs(bit) - 1;
+                if (lo + (double)acc > y) pick = last_pos;
               }
-            };
-            half_walk(m_lo, dm_lo, t_base, 0, tid * W);
-            half_walk(m_hi, dm_hi, t_base + (uint32_t)(n_lo * step), nq_lo, tid * W + 32);
-            *out = pick >= 0 ? pick : last_pos;   // rounding left the sum short: the last id with weight
+            }
           }
-          return true;
-        };
-        if (draws & kDrawResidual) {
-          const double u1 = uniform24(pp.rnd[1]);
-          if (!draw(true, u1, a.cand_res + g)) draw(false, u1, a.cand_res + g);   // a residual without mass
+          // rounding left the sum short: the last id with weight.  No id with weight at all: the
+          // thread's sum was rounding noise of the difference above (about once in 1e8 draws) --
+          // the position goes to the general routines
+          *out = pick >= 0 ? pick : last_pos;
+          if (pick < 0 && last_pos < 0) {
+            atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
+            defer(g);
+          }
         }
-        if (draws & kDrawTarget) draw(false, uniform24(pp.rnd[2]), a.cand_tgt + g);
+        pending &= ~(is_res ? kDrawResidual : kDrawTarget);
+        no_mass = false;
       }
     }
   }
