@@ -90,11 +90,6 @@ struct LanePredictor {
   int dir;
 };
 
-struct LaneCursor {            // next item a warp requests into its ring (phases in consumption order)
-  int left;                    // items still to request
-  int ph, j;                   // phase within the row, row within the parent (0 = draft row)
-  int parent;
-};
 constexpr int kLMaxRows = 17;  // draft row + r*r children, r <= 4
 
 // Selection scratch of one row.  Two copies, used by rows of alternating parity: what a row adds
@@ -107,8 +102,8 @@ struct LaneSel {
   unsigned short sa_owner[kLSetAside];   // the thread whose list holds the entry
   unsigned n_sa;
   unsigned overflow;
-  int w_n[kLWarps];
-  float w_max[kLWarps];
+  unsigned n_total;            // candidates of the row (integer atomics: order-free)
+  unsigned max_key;            // order-preserving key of the row maximum
   double w_e[kLWarps];
   double w_excl[kLWarps];
 };
@@ -122,7 +117,6 @@ struct LanePrep {              // per target row, written by two threads before 
 
 struct LaneSmem {
   uint64_t full[kLWarps][kLStages];   // every warp has a ring of its own
-  LaneCursor cursor[kLWarps];
   LaneSel sel[2];
   LanePrep prep[2];
   double w_tot[2][kLWarps];    // block scan of a draw; consecutive draws alternate
@@ -382,6 +376,8 @@ __global__ void __launch_bounds__(kLThreads, 3)
     for (int s = 0; s < 2; ++s) {
       sm.sel[s].n_sa = 0;
       sm.sel[s].overflow = 0;
+      sm.sel[s].n_total = 0;
+      sm.sel[s].max_key = 0;
       LanePredictor& pr = sm.pred[s];
       pr.have = 0;
       pr.theta = 0.f; pr.rho = 1.f; pr.mx = 0.f;
@@ -406,23 +402,29 @@ __global__ void __launch_bounds__(kLThreads, 3)
     for (int di = 0; di < P.r; ++di)
       for (int dj = 0; dj < P.r; ++dj, ++j) rows[j] = b * N + (ca * P.r + di) * P.W + cc * P.r + dj;
   };
-  auto cursor_issue = [&](LaneCursor& c, int slot) {   // lane 0 of a warp; steps the cursor
-    const uint32_t dst = wring + (uint32_t)slot * kLSlot;
-    uint64_t* bar = &sm.full[warp][slot];
-    const int row = sm.rows[c.parent & 1][c.j];
-    if (c.j == 0) {
-      mbar_expect_tx(bar, kLTile);
-      tma_tile_3d(dst, &tm_q, IDS * c.ph, 32 * warp, row, bar);
-    } else {
-      mbar_expect_tx(bar, HAS_U ? kLSlot : kLTile);
-      tma_tile_3d(dst, &tm_c, IDS * c.ph, 32 * warp, row, bar);
-      if (HAS_U) tma_tile_3d(dst + kLTile, &tm_u, IDS * c.ph, 32 * warp, row, bar);
+  // The next item this warp requests: phase c_ph of row c_j of parent c_par, c_left items to go (the
+  // same in all its lanes; stepping it is a few uniform instructions, the requests are lane 0's).
+  int c_ph = 0, c_j = 0, c_par = p_begin, c_left = (p_end - p_begin) * rows_per_parent * n_ph;
+  auto cursor_issue = [&](int slot) {
+    if (lane == 0) {
+      const uint32_t dst = wring + (uint32_t)slot * kLSlot;
+      uint64_t* bar = &sm.full[warp][slot];
+      const int row = sm.rows[c_par & 1][c_j];
+      if (c_j == 0) {
+        mbar_expect_tx(bar, kLTile);
+        tma_tile_3d(dst, &tm_q, IDS * c_ph, 32 * warp, row, bar);
+      } else {
+        mbar_expect_tx(bar, HAS_U ? kLSlot : kLTile);
+        tma_tile_3d(dst, &tm_c, IDS * c_ph, 32 * warp, row, bar);
+        if (HAS_U) tma_tile_3d(dst + kLTile, &tm_u, IDS * c_ph, 32 * warp, row, bar);
+      }
     }
-    if (++c.ph == n_ph) {
-      c.ph = 0;
-      if (++c.j == rows_per_parent) {
-        c.j = 0;
-        ++c.parent;
+    --c_left;
+    if (++c_ph == n_ph) {
+      c_ph = 0;
+      if (++c_j == rows_per_parent) {
+        c_j = 0;
+        ++c_par;
       }
     }
   };
@@ -431,15 +433,8 @@ __global__ void __launch_bounds__(kLThreads, 3)
     if (p_begin + 1 < p_end) fill_rows(p_begin + 1);
   }
   __syncthreads();
-  if (lane == 0) {
-    const int total = (p_end - p_begin) * rows_per_parent * n_ph;
-    LaneCursor cur;
-    cur.ph = 0; cur.j = 0; cur.parent = p_begin;
-    for (int s = 0; s < kLStages; ++s)
-      if (s < total) cursor_issue(cur, s);
-    cur.left = total > kLStages ? total - kLStages : 0;
-    sm.cursor[warp] = cur;
-  }
+  for (int s = 0; s < kLStages; ++s)
+    if (c_left > 0) cursor_issue(s);
   int rs = 0;   // slots consumed so far: bit 0 = the slot to read next, bit 1 = its phase
 #define rslot (rs & 1)
 #define rphase ((uint32_t)(rs >> 1) & 1u)
@@ -449,14 +444,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
   // one instruction for all lanes; the copy's first write then comes hundreds of cycles later.)
   auto release_slot = [&](uint32_t loaded) {
     asm volatile("" ::"r"(loaded) : "memory");
-    if (lane == 0) {
-      LaneCursor cur = sm.cursor[warp];
-      if (cur.left > 0) {
-        cursor_issue(cur, rslot);
-        --cur.left;
-        sm.cursor[warp] = cur;
-      }
-    }
+    if (c_left > 0) cursor_issue(rslot);
     ++rs;
   };
   auto skip_row = [&]() {
@@ -522,7 +510,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
     const float sd = sqrtf(fmaxf((float)(S2 / cnt) - mean * mean, 1e-20f));
     const float d = fmaxf((a.a_theta - a.a_boot) * sd, 1e-20f);
     pivot = mean + (a.a_boot + pr.shift) * sd;
-    inv_w = (float)kLBins / (2.0f * d);
+    inv_w = (float)kLBins / (3.0f * d);   // (a predicted row's histogram spans 2 d)
     ref = mean + a.a_max * sd;
   };
 
@@ -601,8 +589,8 @@ __global__ void __launch_bounds__(kLThreads, 3)
     const unsigned mk = __reduce_max_sync(kFull, float_key(mx));
     const double es = warp_sum((double)s_all);
     if (lane == 0) {
-      sel.w_n[warp] = nsum;
-      sel.w_max[warp] = key_float(mk);
+      atomicAdd(&sel.n_total, (unsigned)nsum);
+      atomicMax(&sel.max_key, mk);
       sel.w_e[warp] = es;
     }
     return s_all;   // exp of ALL of this thread's entries, in list order
@@ -614,13 +602,8 @@ __global__ void __launch_bounds__(kLThreads, 3)
   };
   // after the barrier that follows pass_one (every warp computes the same)
   auto locate_bin = [&](LaneSel& sel, Sel& s, float ref, int rows) -> bool {
-    int n = 0;
-    float mx = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kLWarps; ++w) {
-      n += sel.w_n[w];
-      mx = fmaxf(mx, sel.w_max[w]);
-    }
+    const int n = (int)sel.n_total;
+    const float mx = key_float(sel.max_key);
     s.n = n;
     s.mx = mx;
     s.reason = 0;
@@ -748,9 +731,11 @@ __global__ void __launch_bounds__(kLThreads, 3)
     const int src = __ffs(hm) - 1;
     th = __shfl_sync(kFull, th, src);
     less_at = __shfl_sync(kFull, less_at, src);
-    double z = 0.0;
+    // the eight warps' partial sums: one per lane, added in a fixed butterfly order
+    double z = lane < kLWarps ? sel.w_e[lane] - sel.w_excl[lane] : 0.0;
 #pragma unroll
-    for (int w = 0; w < kLWarps; ++w) z += sel.w_e[w] - sel.w_excl[w];
+    for (int o = 4; o > 0; o >>= 1) z += __shfl_xor_sync(kFull, z, o);
+    z = __shfl_sync(kFull, z, 0);
     // the bin's entries below theta.  The slots were handed out by atomics in no fixed order, but
     // the sum does not depend on it: the entries of one histogram bin share their exponent (or
     // differ by one), so adding up to 64 fp32 values of that kind in double is exact.
@@ -781,6 +766,8 @@ __global__ void __launch_bounds__(kLThreads, 3)
     if (tid == 0) {
       sel.n_sa = 0;
       sel.overflow = 0;
+      sel.n_total = 0;
+      sel.max_key = 0;
     }
   };
 
