@@ -55,7 +55,9 @@ constexpr int kLRing = kLWarps * kLWarpRing;    // ring bytes of the CTA
 constexpr int kLBins = 256;
 constexpr int kLSetAside = 64;           // entries of the crossing bin that are ranked exactly
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kMaxRefGap = 8.0f;       // a row whose maximum lies further from the exp reference leaves the fast path
+constexpr float kNearRefGap = 8.0f;      // a row whose maximum lies further from the predicted exp reference is summed
+                                         // again against its own maximum (large exponents cost relative accuracy)
+constexpr float kMaxRefGap = 60.0f;      // ... and beyond this the first sum may have left fp32's range: the row is given up
 
 struct LaneArgs {
   DevParams P;
@@ -439,12 +441,17 @@ __global__ void __launch_bounds__(kLThreads, 3)
 #define rslot (rs & 1)
 #define rphase ((uint32_t)(rs >> 1) & 1u)
   static_assert(kLStages == 2, "the packed ring state assumes two slots");
-  // The warp has the slot's words in registers: request the next item into it.  (`loaded` is one
-  // of those words: naming it here makes the request wait for the warp's shared loads, which are
-  // one instruction for all lanes; the copy's first write then comes hundreds of cycles later.)
+  // The warp has the slot's words in registers: request the next item into it.  The lanes of a
+  // warp may drift apart wherever one of them does something alone (the requests below, the
+  // bookkeeping of a failed row); they meet here, before the request -- so that no lane still has
+  // the slot to read -- and after it -- so that none runs on to wait for an item that lane 0 has
+  // not requested yet, or falls a whole barrier phase behind.  (`loaded` is one of the slot's
+  // words: naming it keeps the loads before the meeting point.)
   auto release_slot = [&](uint32_t loaded) {
     asm volatile("" ::"r"(loaded) : "memory");
+    __syncwarp();
     if (c_left > 0) cursor_issue(rslot);
+    __syncwarp();
     ++rs;
   };
   auto skip_row = [&]() {
@@ -594,6 +601,18 @@ __global__ void __launch_bounds__(kLThreads, 3)
       sel.w_e[warp] = es;
     }
     return s_all;   // exp of ALL of this thread's entries, in list order
+  };
+
+  // a row whose maximum turned out far from the predicted reference: the sum once more, against
+  // the maximum itself (between the row's first and second barrier)
+  auto sum_again = [&](LaneSel& sel, uint32_t base, int n, float c0) -> float {
+    float s_all = 0.f;
+    uint32_t ad = base;
+#pragma unroll 1
+    for (int i = 0; i < n; ++i, ad += step) s_all += ex2f(fmaf(lds_f32(ad), kLog2e, c0));
+    const double es = warp_sum((double)s_all);
+    if (lane == 0) sel.w_e[warp] = es;
+    return s_all;
   };
 
   struct Sel {
@@ -791,7 +810,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
       const int t = (int)g - pb * N;
       float pivot, inv_w, ref;
       choose_pivot(is_q ? 0 : 1, HAS_U && !is_q, pivot, inv_w, ref);
-      const float c0 = -ref * kLog2e;
+      float c0 = -ref * kLog2e;
       // Two threads prepare what the row needs besides its lists: the logit of x~ (requested here by
       // asynchronous copies, read after the row has been streamed, so that no warp sits on the load)
       // and the position's uniforms.
@@ -841,6 +860,11 @@ __global__ void __launch_bounds__(kLThreads, 3)
         if (tid == 64 && parent + 1 < p_end && parent > p_begin) fill_rows(parent + 1);
       }
       float s_inc = s_all;   // becomes: exp of this thread's entries that are >= theta
+      if (ok && !(fabsf(s.mx - ref) <= kNearRefGap)) {   // block-uniform, rare
+        c0 = -s.mx * kLog2e;
+        s_inc = sum_again(sel, base, n, c0);
+        if (tid == kLThreads - 1 && !is_q) pp.e_tok = lane_exp2((double)pp.z_tok * (double)kLog2e + (double)c0);
+      }
       if (ok) s_inc -= set_aside(sel, base, lowm, pivot, inv_w, c0, s.bstar);
       __syncthreads();   // ---- barrier 2
       float theta = 0.f;
