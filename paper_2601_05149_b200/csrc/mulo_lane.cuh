@@ -86,6 +86,7 @@ struct LaneArgs {
 // running prediction for one kind of row (draft / target), per CTA
 struct LanePredictor {
   int have;
+  int age;                    // rows learnt from since the prediction was last lost
   float theta, rho, mx;       // running k-th largest, density below it, row maximum
   float pivot, inv_w, ref;    // what the next row starts from (valid while have != 0)
   float shift, step;          // bootstrap adaptation, as in the general streaming kernel
@@ -300,6 +301,7 @@ __device__ __noinline__ void lane_learn(LanePredictor* prp, bool ok, int reason,
   LanePredictor pr = *prp;
   if (!ok) {
     pr.have = 0;
+    pr.age = 0;
     const int dir = reason == 2 ? -1 : (reason == 1 || reason == 3) ? 1 : 0;
     if (dir != 0) {
       const float unit = 0.5f * (a_theta - a_boot);
@@ -312,21 +314,27 @@ __device__ __noinline__ void lane_learn(LanePredictor* prp, bool ok, int reason,
   } else {
     pr.dir = 0;
     const int below = n - n_ge;   // candidates in [pivot, theta)
+    // running means: a plain average over the first four rows, weight 1/4 for the newest after that
+    const float w_new = pr.have ? fmaxf(0.25f, 1.0f / (float)(pr.age + 1)) : 1.0f;
     float rho = pr.rho;
     bool rho_ok = pr.have != 0;
     if (theta > pivot && below >= 16) {
       const float r_new = (float)below / (theta - pivot);
-      rho = pr.have ? pr.rho + 0.25f * (r_new - pr.rho) : r_new;
+      rho = pr.have ? pr.rho + w_new * (r_new - pr.rho) : r_new;
       rho_ok = true;
     }
     if (!rho_ok) {
       pr.have = 0;
+      pr.age = 0;
     } else {
-      pr.theta = pr.have ? pr.theta + 0.25f * (theta - pr.theta) : theta;
-      pr.mx = pr.have ? pr.mx + 0.25f * (mx - pr.mx) : mx;
+      pr.theta = pr.have ? pr.theta + w_new * (theta - pr.theta) : theta;
+      pr.mx = pr.have ? pr.mx + w_new * (mx - pr.mx) : mx;
       pr.rho = rho;
       pr.have = 1;
-      const float d = (float)margin / rho;
+      if (pr.age < 8) ++pr.age;
+      // a prediction that rests on a single row carries that row's noise in the threshold and in
+      // the density: the row after it aims for a wider margin
+      const float d = (pr.age < 2 ? 1.4f : 1.0f) * (float)margin / rho;
       pr.pivot = pr.theta - d;
       pr.inv_w = (float)kLBins / (2.0f * d);   // the histogram spans twice the distance pivot -> threshold
       pr.ref = pr.mx;
@@ -356,15 +364,20 @@ __global__ void __launch_bounds__(kLThreads, 3)
   // ---- this thread's places in shared memory
   // (the swizzle works on address bits 4 and 7: the ring starts on a 256-byte boundary)
   const uint32_t ring = (smem_u32(dyn) + 255u) & ~255u;
-  // A list column (R rows of 512 bytes; lane l of a warp sits in bank l) belongs to threads t and
-  // t + 128 and holds four stacks: the draft row's entries of t from row 0 upwards and of t + 128
-  // from row R - 1 downwards (fixed while the parent's children are verified), and between them the
-  // current target row's entries of the two threads, again growing towards each other.  A stack is
-  // clamped at the first row of the stack it grows towards, so it can never reach the draft entries
-  // of the other thread; whether two stacks met is checked from the four counts.
+  // A list column (R rows of 512 bytes; lane l of a warp sits in bank l) holds four stacks: the
+  // draft row's entries of thread c from row 0 upwards and of c + 128 from row R - 1 downwards (fixed
+  // while the parent's children are verified), and between them the current target row's entries
+  // of two OTHER threads, c ^ 64 and (c ^ 64) + 128, again growing towards each other.  (A thread's
+  // draft and target entries cover the same ids and their counts rise and fall together, the target
+  // rows being the draft row plus noise: four stacks of four different id ranges overflow far more
+  // rarely than two pairs.)  A stack is clamped at the first row of the stack it grows towards, so
+  // it can never reach the draft entries at the column's other end; whether the two target stacks
+  // met is checked from the four counts.
   const bool up = tid < kLThreads / 2;
   const int step = up ? 512 : -512;
-  const uint32_t col = ring + kLRing + (uint32_t)(tid & 127) * 4u;
+  const int colq = tid & 127, colt = colq ^ 64;   // the columns of this thread's draft / target stack
+  const uint32_t col = ring + kLRing + (uint32_t)colq * 4u;
+  const uint32_t tcol = ring + kLRing + (uint32_t)colt * 4u;
   const uint32_t q_base = col + (up ? 0u : (uint32_t)(R - 1) * 512u);
   const uint32_t q_lim = col + (up ? (uint32_t)(R - 1) * 512u : 0u);   // the partner's first draft row
   const uint32_t sw = ((uint32_t)lane >> 2) & 1u;          // 32-byte swizzle: address bit 4 ^= bit 7
@@ -382,6 +395,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
       sm.sel[s].max_key = 0;
       LanePredictor& pr = sm.pred[s];
       pr.have = 0;
+      pr.age = 0;
       pr.theta = 0.f; pr.rho = 1.f; pr.mx = 0.f;
       pr.pivot = 0.f; pr.inv_w = 0.f; pr.ref = 0.f;
       pr.shift = 0.f; pr.step = 0.f; pr.dir = 0;
@@ -791,7 +805,8 @@ __global__ void __launch_bounds__(kLThreads, 3)
   };
 
   uint32_t dm_lo = 0, dm_hi = 0;   // survivor mask of the parent's draft row (this thread's ids)
-  int nq = 0, nq_other = 0;        // draft entries of this thread and of the thread it shares the column with
+  int nq = 0;                      // draft entries of this thread
+  int nq_up = 0, nq_dn = 0;        // draft entries at the two ends of the column that takes its target entries
   int rowi = 0;                    // rows done by this CTA (its parity selects the scratch copies)
 
   if (tid == kLThreads - 1) sm.tok[p_begin & 1] = __ldg(a.draft_tok_lo + p_begin);
@@ -808,6 +823,9 @@ __global__ void __launch_bounds__(kLThreads, 3)
       ++rowi;
       const size_t g = (size_t)sm.rows[parent & 1][j];   // a target row's position b * N + t (the draft row's cell)
       const int t = (int)g - pb * N;
+      // a draft row's entries go where other threads kept the previous parent's target entries: the
+      // thread that walked the last draw must be done with them
+      if (is_q && parent > p_begin) __syncthreads();
       float pivot, inv_w, ref;
       choose_pivot(is_q ? 0 : 1, HAS_U && !is_q, pivot, inv_w, ref);
       float c0 = -ref * kLog2e;
@@ -835,8 +853,9 @@ __global__ void __launch_bounds__(kLThreads, 3)
       }
       // where the row's entries go: the draft row's from the end of the column, a target row's from
       // the end of the thread's draft entries, up to the first target row of the other thread
-      const uint32_t base = is_q ? q_base : q_base + (uint32_t)(nq * step);
-      const uint32_t lim = is_q ? q_lim : q_lim - (uint32_t)(nq_other * step);
+      const uint32_t t_first = tcol + (uint32_t)nq_up * 512u, t_last = tcol + (uint32_t)(R - 1 - nq_dn) * 512u;
+      const uint32_t base = is_q ? q_base : up ? t_first : t_last;
+      const uint32_t lim = is_q ? q_lim : up ? t_last : t_first;
       uint32_t m_lo, m_hi;
       const int n = stream_row(sel, HAS_U && !is_q, base, lim, pivot, m_lo, m_hi);
       uint32_t lowm;
@@ -852,9 +871,10 @@ __global__ void __launch_bounds__(kLThreads, 3)
       __syncthreads();   // ---- barrier 1
       reset_selection(sm.sel[rowi & 1]);
       Sel s;
-      bool ok = locate_bin(sel, s, ref, is_q ? R : R - nq - nq_other);
+      bool ok = locate_bin(sel, s, ref, is_q ? R : R - nq_up - nq_dn);
       if (is_q) {
-        nq_other = sm.cnt[tid ^ 128];
+        nq_up = sm.cnt[colt];
+        nq_dn = sm.cnt[colt + 128];
         // the warps are requesting rows of this parent and (at its end) of the next; the table entry of
         // the parent after that replaces the previous parent's, whose last request is behind every warp
         if (tid == 64 && parent + 1 < p_end && parent > p_begin) fill_rows(parent + 1);
@@ -926,11 +946,14 @@ __global__ void __launch_bounds__(kLThreads, 3)
         __syncthreads();   // the predictor
         continue;
       }
-      {   // this thread's entries of the crossing bin that fell below theta
+      {   // this thread's entries of the crossing bin that fell below theta (their slots were handed
+          // out in no fixed order: summed in double, which is exact for values of one bin, the
+          // result does not depend on it)
         const int mcount = (int)sel.n_sa;
+        double mine = 0.0;
         for (int i = 0; i < mcount; ++i)
-          if (sel.sa_owner[i] == tid && sel.sa_z[i] < theta) s_inc -= sel.sa_e[i];
-        s_inc = fmaxf(s_inc, 0.f);
+          if (sel.sa_owner[i] == tid && sel.sa_z[i] < theta) mine += (double)sel.sa_e[i];
+        s_inc = fmaxf((float)((double)s_inc - mine), 0.f);
       }
       // ---- the decision (Eq. 1 / Eq. 5), the same in every thread
       const double e_tok = (pp.z_tok >= theta) ? pp.e_tok : 0.0;

@@ -304,8 +304,10 @@ def test_config_C4_sampled_images(ctx):
     batch = pu.build_batch(cfg)
     for radius in (3, 1, 2):
         c = dataclasses.replace(cfg, radius=radius)
+        ctx.poll_fallback_counts()
         g = pu.gpu_round(ctx, c, batch, probs=(radius == 3))
-        assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
+        assert ctx.poll_device_status() == 0
+        assert ctx.poll_fallback_counts()[0] == 0      # no row left the fast path
         if radius == 3:
             o = pu.oracle_images(c, batch, [0, cfg.B - 1])
         else:   # only the masks and the choice of draw depend on the radius
@@ -313,14 +315,29 @@ def test_config_C4_sampled_images(ctx):
         pu.check_round(c, g, o)
 
 
-@pytest.mark.parametrize("pick", [0, 43, 95], ids=["32x32-V8192-s0.1", "64x64-V8192-s2.0", "96x96-V16384-s2.0"])
-def test_sweep_points_sampled(ctx, pick):
-    """Points of the throughput sweep (batch cut to 2 images to bound the oracle's time)."""
-    cfg = dataclasses.replace(synth.sweep_points()[pick], B=2)
+def _sweep_picks():
+    """Twelve points of the throughput sweep at its largest batch: every (grid, vocabulary) pair twice,
+    every noise level three times."""
+    pts = synth.sweep_points()
+    picks = []
+    for pair in range(6):               # (grid, V) pairs in the sweep's own order
+        for s in ((2 * pair) % 4, (2 * pair + 1) % 4):
+            picks.append((pair * 4 + 3) * 4 + s)     # batch index 3: B = 64
+    return [pts[i] for i in picks]
+
+
+@pytest.mark.parametrize("cfg", _sweep_picks(), ids=lambda c: f"{c.H}x{c.W}-V{c.V}-B{c.B}-s{c.sigma}")
+def test_sweep_points_at_launch_size(ctx, cfg):
+    """Points of the throughput sweep in the configuration the sweep times (B = 64 on the device): the
+    first four images and the last against the oracle, no row redone by the general kernel."""
+    assert cfg.B == 64
     batch = pu.build_batch(cfg)
+    ctx.poll_fallback_counts()
     g = pu.gpu_round(ctx, cfg, batch)
-    assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
-    o = pu.oracle_images(cfg, batch, [1])
+    counts = ctx.poll_fallback_counts()      # rows redone, then by reason: list full, too few, above range, crowded bin
+    assert counts[0] == 0, counts
+    assert ctx.poll_device_status() == 0
+    o = pu.oracle_images(cfg, batch, [0, 1, 2, 3, cfg.B - 1])
     pu.check_round(cfg, g, o)
 
 
@@ -429,3 +446,67 @@ def test_round_replays_from_a_cuda_graph(ctx):
     for k in direct:
         assert torch.equal(direct[k], replay[k]), k
     assert int(direct["n_reject"].sum()) > 0
+
+
+@pytest.mark.parametrize("fast", [True, False], ids=["fast-path", "general-path"])
+def test_draft_token_without_draft_mass(ctx, fast):
+    """q(x~) = 0: the drafter's token lies outside the draft row's own top-k set at a few cells (a
+    contract violation the round must survive).  Eq. 1 then accepts iff p(x~) > 0; decisions, masks
+    and tokens follow the oracle on both kernels, and the status bit is raised."""
+    cfg = dataclasses.replace(BIG, V=4096, top_k=500, H=16, W=16, radius=2, seed=260)
+    batch = pu.build_batch(cfg)
+    tok = batch["tok_lo"].clone()
+    cells = [(0, 0, 0), (0, 3, 5), (1, 7, 7), (1, 2, 0)]
+    order = batch["draft_lo"].float().argsort(-1)
+    for n, (b, i, j) in enumerate(cells):
+        # the draft row's least likely id, and (last two cells) one just outside its top-k set
+        tok[b, i, j] = order[b, i, j, 0] if n < 2 else order[b, i, j, cfg.V - cfg.top_k - 1 - n]
+    batch["tok_lo"] = tok.contiguous()
+    ctx.poll_device_status()
+    ctx.set_general_path_only(not fast)
+    try:
+        n0 = ctx.kernel_launches()
+        g = pu.gpu_round(ctx, cfg, batch)
+        assert (ctx.kernel_launches() - n0 == 3) == fast
+    finally:
+        ctx.set_general_path_only(False)
+    status = ctx.poll_device_status()
+    assert status & binding.DEV_ZERO_DRAFT_PROB and status & ~(binding.DEV_ZERO_DRAFT_PROB | binding.DEV_DENSE_FALLBACK) == 0
+    o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
+    pu.check_round(cfg, g, o)
+    for (b, i, j) in cells:
+        for di in range(cfg.r):
+            for dj in range(cfg.r):
+                y, x = i * cfg.r + di, j * cfg.r + dj
+                assert g["q_tok"][b, y, x] == 0.0 and o[b]["q_tok"][y, x] == 0.0
+                # accepted iff the target gives the token any mass; the threshold is then 1 or 0
+                assert g["accept_prob"][b, y, x] == (1.0 if o[b]["p_tok"][y, x] > 0 else 0.0)
+                assert g["reject"][b, y, x] == (0 if o[b]["p_tok"][y, x] > 0 else 1)
+
+
+def test_round_is_bit_reproducible_at_launch_size(ctx):
+    """The benchmark's workload (B = 32): the same call twice, and once more from another stream,
+    gives every output array bit for bit -- decisions depend on (seed, image, position, round) and the
+    inputs only, not on how CTAs were scheduled."""
+    cfg = synth.CONFIGS["C4"]
+    batch = pu.build_batch(cfg)
+    p = binding.params_from_config(cfg)
+    ctx.ensure_workspace(p)
+
+    def run(stream):
+        o, guard = pu.round_outputs(p, "cuda", True)
+        ctx.mulo_round(p, batch["cond"], batch["uncond"], batch["draft_lo"], batch["tok_lo"], batch["nn"],
+                       o["out_tok"], o["reject_bits"], o["expand_bits"], o["p_tok"], o["q_tok"], o["accept_prob"],
+                       o["n_reject"], o["n_expand"], o["first_reject"], stream=stream)
+        torch.cuda.synchronize()
+        guard.check()
+        return {k: v.cpu().numpy() for k, v in o.items()}
+
+    first = run(None)
+    second = run(None)
+    side = torch.cuda.Stream()
+    third = run(side)
+    for k in first:
+        assert first[k].tobytes() == second[k].tobytes(), k
+        assert first[k].tobytes() == third[k].tobytes(), k
+    assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
