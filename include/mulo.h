@@ -58,7 +58,8 @@ typedef enum {
   MULO_ERR_UNSUPPORTED = 2, /* valid but outside what the kernels handle (see limits)   */
   MULO_ERR_WORKSPACE = 3,   /* no workspace set, or too small for these parameters      */
   MULO_ERR_CUDA = 4,        /* a CUDA runtime call failed (also: no usable device)      */
-  MULO_ERR_TIMEOUT = 5      /* reserved for bounded device-side waits; unused today     */
+  MULO_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (MULO_DEV_TIMEOUT): the
+                               results of the calls since the last poll are invalid     */
 } mulo_status;
 
 typedef enum { MULO_F32 = 0, MULO_BF16 = 1 } mulo_dtype;
@@ -125,8 +126,16 @@ mulo_status mulo_workspace_bytes(const mulo_params* p, size_t* bytes);
  * and must not be shared by calls that overlap on the device.  The first 256 bytes hold
  * the device status word; this call clears it (on the default stream, synchronously). */
 mulo_status mulo_set_workspace(mulo_ctx* ctx, void* dev_ptr, size_t bytes);
-/* Synchronises `stream`, reads and clears the device status bits (MULO_DEV_*). */
+/* Synchronises `stream`, reads and clears the device status bits (MULO_DEV_*).  *flags is
+ * written in every case that got as far as reading them; the return value is
+ * mulo_status_of_device_flags(*flags): MULO_ERR_TIMEOUT if a kernel's bounded wait on one of
+ * its own copies gave up.  A CTA whose wait gave up writes nothing further (its remaining
+ * rows keep whatever the workspace held), waits a bounded time for its copies in flight and
+ * returns; the other CTAs finish.  The context stays usable. */
 mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags);
+/* The status that a set of device status bits maps to (host arithmetic only): MULO_ERR_TIMEOUT
+ * if MULO_DEV_TIMEOUT is among them, else MULO_OK -- the other bits are reports, not errors. */
+mulo_status mulo_status_of_device_flags(uint32_t flags);
 /* Synchronises `stream`, reads and clears five counters kept next to the status bits:
  * counts[0] rows that mulo_round's fast kernel handed to the general routines, and of those
  * counts[1] because a candidate list was full, counts[2] because fewer than top_k candidates
@@ -138,11 +147,20 @@ mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags
 mulo_status mulo_poll_fallback_counts(mulo_ctx* ctx, void* stream, uint32_t counts[5]);
 /* Number of kernels this context has launched so far. */
 mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
-/* mulo_round and mulo_sample_draft pick between two row kernels: a fast one for rows with
- * top-k on (V >= 1024; with pooling, V <= 16384; each row streamed once, work done on the few
- * thousand entries near and above the top-k threshold; a row it cannot handle is redone by
- * the general routines) and the general one.  Both compute the same function.  `on` != 0
- * makes this context always use the general kernel (for testing and comparison). */
+/* mulo_round picks between three row kernels, mulo_sample_draft between the last two.  All
+ * compute the same function; a row a fast kernel cannot handle is redone by the general routines.
+ *   MULO_KERNEL_LANE     top-k on, pooling off, V a multiple of 4096 (bf16) or 2048 (fp32) and
+ *                        at most 16384: every thread of a CTA owns a contiguous range of the
+ *                        vocabulary, rows are streamed once through per-warp shared-memory rings;
+ *   MULO_KERNEL_STREAM   top-k on, V >= 1024 (with pooling, V <= 16384), any other shape: rows
+ *                        streamed once in chunks, candidates compacted per segment;
+ *   MULO_KERNEL_GENERAL  everything else (top-k off, tiny vocabularies): one CTA per row, the
+ *                        row read several times (from L2 after the first).
+ * mulo_round_kernel reports the choice for these parameters on this context (host arithmetic
+ * only; nothing is launched).  mulo_set_general_path_only(on != 0) makes the context always use
+ * the general kernel (for testing and comparison). */
+typedef enum { MULO_KERNEL_GENERAL = 0, MULO_KERNEL_STREAM = 1, MULO_KERNEL_LANE = 2 } mulo_kernel;
+mulo_status mulo_round_kernel(const mulo_ctx* ctx, const mulo_params* p, int* kernel);
 mulo_status mulo_set_general_path_only(mulo_ctx* ctx, int on);
 /* Optional device timing of the fused row kernel (the launch that reads the logits):
  * mulo_set_timing prepares CUDA event pairs for up to max_launches (<= 4096) calls of

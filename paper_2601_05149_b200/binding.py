@@ -22,8 +22,9 @@ DEV_ZERO_DRAFT_PROB, DEV_BAD_TOKEN, DEV_DENSE_FALLBACK, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = (
     "mulo_create", "mulo_destroy", "mulo_status_string", "mulo_workspace_bytes",
-    "mulo_set_workspace", "mulo_poll_device_status", "mulo_poll_fallback_counts", "mulo_kernel_launches",
-    "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only",
+    "mulo_set_workspace", "mulo_poll_device_status", "mulo_status_of_device_flags", "mulo_poll_fallback_counts",
+    "mulo_kernel_launches",
+    "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only", "mulo_round_kernel",
     "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_islands", "mulo_island_schedule", "mulo_sample_draft", "mulo_downsample", "mulo_resample",
     "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host", "mulo_round_static",
 )
@@ -78,6 +79,11 @@ def lib() -> C.CDLL:
                 fn.restype = C.c_int
         _lib = L
     return _lib
+
+
+def status_of_device_flags(flags: int) -> int:
+    """The status a set of MULO_DEV_* bits maps to (ERR_TIMEOUT or OK)."""
+    return lib().mulo_status_of_device_flags(C.c_uint32(flags))
 
 
 def status_string(status: int) -> str:
@@ -170,9 +176,14 @@ class Context:
             self.set_workspace(torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}"))
 
     def poll_device_status(self, stream=None) -> int:
+        """The MULO_DEV_* bits since the last poll; raises MuloError(ERR_TIMEOUT) if a kernel's
+        bounded wait gave up (the bits are then in the exception's ``flags``)."""
         f = C.c_uint32()
-        _check(lib().mulo_poll_device_status(self._ctx, _stream(stream), C.byref(f)),
-               "mulo_poll_device_status")
+        st = lib().mulo_poll_device_status(self._ctx, _stream(stream), C.byref(f))
+        if st != OK:
+            e = MuloError(st, "mulo_poll_device_status")
+            e.flags = f.value
+            raise e
         return f.value
 
     def poll_fallback_counts(self, stream=None):
@@ -186,6 +197,12 @@ class Context:
         n = C.c_uint64()
         _check(lib().mulo_kernel_launches(self._ctx, C.byref(n)), "mulo_kernel_launches")
         return n.value
+
+    def round_kernel(self, p: "MuloParams") -> str:
+        """The row kernel ``mulo_round`` launches for these parameters: "lane", "stream" or "general"."""
+        k = C.c_int()
+        _check(lib().mulo_round_kernel(self._ctx, C.byref(p), C.byref(k)), "mulo_round_kernel")
+        return ("general", "stream", "lane")[k.value]
 
     def set_general_path_only(self, on: bool):
         _check(lib().mulo_set_general_path_only(self._ctx, int(bool(on))), "mulo_set_general_path_only")

@@ -642,6 +642,10 @@ mulo_status mulo_set_workspace(mulo_ctx* ctx, void* dev_ptr, size_t bytes) {
   return MULO_OK;
 }
 
+mulo_status mulo_status_of_device_flags(uint32_t flags) {
+  return (flags & MULO_DEV_TIMEOUT) ? MULO_ERR_TIMEOUT : MULO_OK;
+}
+
 mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags) {
   if (!ctx || !flags) return MULO_ERR_INVALID_ARG;
   if (!ctx->ws) return MULO_ERR_WORKSPACE;
@@ -649,7 +653,7 @@ mulo_status mulo_poll_device_status(mulo_ctx* ctx, void* stream, uint32_t* flags
   if (cudaMemcpyAsync(flags, ctx->ws, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MULO_ERR_CUDA;
   if (cudaMemsetAsync(ctx->ws, 0, sizeof(uint32_t), st) != cudaSuccess) return MULO_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MULO_ERR_CUDA;
-  return MULO_OK;
+  return mulo_status_of_device_flags(*flags);
 }
 
 mulo_status mulo_poll_fallback_counts(mulo_ctx* ctx, void* stream, uint32_t counts[5]) {
@@ -1219,6 +1223,22 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   m.draft_tok_lo = draft_tok_lo; m.out_tok = out_tok;
   k_mask<2><<<p->B, kMaskThreads, mask_smem(p), st>>>(m);
   return launched(ctx, fast ? 3 : 2);
+}
+
+mulo_status mulo_round_kernel(const mulo_ctx* ctx, const mulo_params* p, int* kernel) {
+  if (!ctx || !kernel) return MULO_ERR_INVALID_ARG;
+  const mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  const DevParams d = to_dev(p);
+  LaneArgs la;
+  StreamArgs sa;
+  memset(&la, 0, sizeof la);
+  memset(&sa, 0, sizeof sa);
+  *kernel = MULO_KERNEL_GENERAL;
+  if (ctx->force_dense) return MULO_OK;
+  if (!ctx->no_lane && plan_lane(ctx, d, &la)) *kernel = MULO_KERNEL_LANE;
+  else if (plan_stream(ctx, d, &sa)) *kernel = MULO_KERNEL_STREAM;
+  return MULO_OK;
 }
 
 // ---- host-buffer variant -------------------------------------------------------------

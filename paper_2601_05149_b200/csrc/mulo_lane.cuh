@@ -131,6 +131,7 @@ struct LaneSmem {
   int tok[2];                  // the draft token of the parent in work / of the next one
   int rows[2][kLMaxRows];      // row index (within its tensor) of every row of a parent, by parent parity
   int image[2];                // image index of the parent, by parent parity
+  int abort;                   // a wait of this CTA gave up: stop at the next row's first barrier
 };
 
 __device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint64_t* bar) {
@@ -139,13 +140,17 @@ __device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap* tm,
       "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
       : "memory");
 }
-// Bounded wait on a ring slot: after kSpinLimit tries the wait gives up and raises the time-out bit.
-__device__ __forceinline__ void lane_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status) {
+// Bounded wait on a ring slot: after kSpinLimit tries the wait gives up, raises the time-out bit
+// and the CTA's abort flag; once that flag is up every later wait of the CTA returns at once, and
+// the CTA stops at the next row's first barrier.
+__device__ __forceinline__ void lane_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status, volatile int* abort) {
   if (mbar_try_wait(bar, parity)) return;
+  if (*abort) return;
 #pragma unroll 1
   for (uint32_t it = 0; it < kSpinLimit; ++it)
     if (mbar_try_wait(bar, parity)) return;
   atomicOr(dev_status, MULO_DEV_TIMEOUT);
+  *abort = 1;
 }
 // 4-byte asynchronous global -> shared copy (no register holds the value while it is in flight)
 __device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
@@ -388,6 +393,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
     for (int w = 0; w < kLWarps; ++w)
       for (int s = 0; s < kLStages; ++s) mbar_init(&sm.full[w][s], 1);
     mbar_fence_init();
+    sm.abort = 0;
     for (int s = 0; s < 2; ++s) {
       sm.sel[s].n_sa = 0;
       sm.sel[s].overflow = 0;
@@ -470,7 +476,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
   };
   auto skip_row = [&]() {
     for (int ph = 0; ph < n_ph; ++ph) {
-      lane_wait(&sm.full[warp][rslot], rphase, a.dev_status);
+      lane_wait(&sm.full[warp][rslot], rphase, a.dev_status, &sm.abort);
       release_slot(0u);
     }
   };
@@ -486,7 +492,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
     const LanePredictor pr = sm.pred[kind];
     // no prediction: mean and spread of the row's first phase (every thread's first ids: an
     // even sample of the row), assuming a normal shape; the slot is read again by the dense pass
-    lane_wait(&sm.full[warp][rslot], rphase, a.dev_status);
+    lane_wait(&sm.full[warp][rslot], rphase, a.dev_status, &sm.abort);
     const uint32_t sb = wring + (uint32_t)rslot * kLSlot + my_off;
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
@@ -546,7 +552,7 @@ __global__ void __launch_bounds__(kLThreads, 3)
     m_hi = 0;
 #pragma unroll 1
     for (int ph = 0; ph < n_ph; ++ph) {
-      lane_wait(&sm.full[warp][rslot], rphase, a.dev_status);
+      lane_wait(&sm.full[warp][rslot], rphase, a.dev_status, &sm.abort);
       const uint32_t room = (up ? lim - cur : cur - lim) >> 9;   // rows between the cursor and the other stack
       uint32_t stp = (uint32_t)step;
       if (room < (uint32_t)IDS) {
@@ -869,6 +875,16 @@ __global__ void __launch_bounds__(kLThreads, 3)
         pp.e_tok = lane_exp2((double)z * (double)kLog2e + (double)c0);   // the list entries' own exponent
       }
       __syncthreads();   // ---- barrier 1
+      if (*(volatile int*)&sm.abort) {   // block-uniform: the flag was raised before the barrier
+        // Nothing more is written for this CTA's rows (the status bit says that the call's results
+        // are invalid).  Before its shared memory is given up, every warp waits -- bounded again --
+        // for the copies it still has in flight: the items it requested and did not consume.
+        const int issued = (p_end - p_begin) * rows_per_parent * n_ph - c_left;
+        for (; rs < issued; ++rs)
+          for (uint32_t it = 0; it < (1u << 16); ++it)
+            if (mbar_try_wait(&sm.full[warp][rslot], rphase)) break;
+        return;
+      }
       reset_selection(sm.sel[rowi & 1]);
       Sel s;
       bool ok = locate_bin(sel, s, ref, is_q ? R : R - nq_up - nq_dn);

@@ -69,11 +69,16 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
 
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded waits: give up, flag, carry on
 
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status) {
+// After a wait has given up, the CTA's abort flag is up: later waits return at once and the
+// CTA stops at its next parent (the data is garbage by then, but nothing hangs).
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return;
+  if (*abort) return;
 #pragma unroll 1
   for (uint32_t it = 0; it < kSpinLimit; ++it)
     if (mbar_try_wait(bar, parity)) return;
-  atomicOr(dev_status, MULO_DEV_TIMEOUT);   // the data is then garbage, but nothing hangs
+  atomicOr(dev_status, MULO_DEV_TIMEOUT);
+  *abort = 1;
 }
 
 // two fp32 operations per instruction (sm_100 packed fp32); each half is the
@@ -238,6 +243,7 @@ struct StreamSmem {
   int b, ca, cc;
   // the parent the address table was last filled for
   int tb, tca, tcc, tparent;
+  int abort;           // a wait of this CTA gave up
   unsigned long long row_off[kTableParents][kMaxRowsPerParent];   // byte offsets of the rows within their tensors
 };
 
@@ -491,6 +497,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       sm.done[s] = 0;
     }
     mbar_fence_init();
+    sm.abort = 0;
     rs.n_cand = 0;
     rs.n_member = 0;
     rs.overflow = 0;
@@ -586,7 +593,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       inv_w = pr.inv_w;
       return;
     }
-    mbar_wait(&sm.full[rslot], rphase, a.dev_status);
+    mbar_wait(&sm.full[rslot], rphase, a.dev_status, &sm.abort);
     const unsigned char* slot = ring + (size_t)rslot * a.slot_bytes;
     const int elems = min(a.chunk, P.V);
     float s1 = 0.f, s2 = 0.f;
@@ -629,7 +636,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
   // that left the fast path).
   auto skip_row = [&]() {
     for (int c = 0; c < a.n_chunks; ++c) {
-      mbar_wait(&sm.full[rslot], rphase, a.dev_status);
+      mbar_wait(&sm.full[rslot], rphase, a.dev_status, &sm.abort);
       release_slot();
     }
   };
@@ -642,7 +649,7 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
     constexpr bool ROW_U = decltype(has_u_tag)::value;
     ushort2* const run = IS_Q ? qseg : tseg;
     for (int c = 0; c < a.n_chunks; ++c) {
-      mbar_wait(&sm.full[rslot], rphase, a.dev_status);
+      mbar_wait(&sm.full[rslot], rphase, a.dev_status, &sm.abort);
       const unsigned char* slot = ring + (size_t)rslot * a.slot_bytes;
       uint4 rc[kPPW], ru[kPPW];
 #pragma unroll
@@ -1126,6 +1133,12 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       choose_pivot(0, std::false_type{}, pivot, inv_w);
       stream_row(std::true_type{}, std::false_type{}, pivot, inv_w);
       __syncthreads();
+      if (*(volatile int*)&sm.abort) {   // block-uniform: raised before the barrier
+        // nothing more is written for this CTA's rows; its copies in flight (at most kStages chunks)
+        // get a bounded time to land before the shared memory is given up
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        return;
+      }
       if (!SAMPLE && tid == 64) prefetch_row(0);
       Sel s;
       bool ok = locate_bin(s);

@@ -133,19 +133,6 @@ def make_image(cfg: RoundConfig, b: int, device="cpu"):
                 uncond=None if uncond is None else uncond.contiguous())
 
 
-def draw_draft_tokens(cfg: RoundConfig, b: int, draft_lo: torch.Tensor) -> torch.Tensor:
-    """One token per low-res cell, drawn from the drafter's distribution
-    (temperature, top-k with ties kept) -- int32 ``[h, w]``."""
-    g = _gen(replace(cfg, seed=cfg.seed + 7919), b, draft_lo.device)
-    z = draft_lo.float().reshape(-1, cfg.V) / cfg.temperature
-    if 0 < cfg.top_k < cfg.V:
-        kth = torch.topk(z, cfg.top_k, dim=-1).values[:, -1:]
-        z = z.masked_fill(z < kth, float("-inf"))
-    prob = torch.softmax(z, dim=-1)
-    tok = torch.multinomial(prob, 1, generator=g).reshape(cfg.h, cfg.w)
-    return tok.to(torch.int32).contiguous()
-
-
 def codebook_neighbours(V: int, k: int, seed: int, device="cpu") -> torch.Tensor:
     """``[V, k]`` uint16-valued ids (returned as int32 holding 0..V-1, cast by the
     caller): the k nearest entries of a random 8-dim codebook, self first."""
@@ -178,19 +165,21 @@ def neighbours_to_numpy(nn: torch.Tensor) -> np.ndarray:
 
 
 def build_batch(cfg: RoundConfig, device="cuda"):
-    """All inputs of one round as device tensors."""
+    """The logits of one round as device tensors, and an UNFILLED ``tok_lo`` [B, h, w] int32: the
+    drafter's tokens are the caller's to draw (this module holds none of the method's arithmetic) --
+    with ``mulo_sample_draft`` in the benchmark and the round driver, with the oracle's sampler
+    where the tokens feed the oracle."""
     dt = cfg.torch_dtype
     cond = torch.empty((cfg.B, cfg.H, cfg.W, cfg.V), dtype=dt, device=device)
     uncond = torch.empty_like(cond) if cfg.has_uncond else None
     draft = torch.empty((cfg.B, cfg.h, cfg.w, cfg.V), dtype=dt, device=device)
-    tok = torch.empty((cfg.B, cfg.h, cfg.w), dtype=torch.int32, device=device)
+    tok = torch.zeros((cfg.B, cfg.h, cfg.w), dtype=torch.int32, device=device)
     for b in range(cfg.B):
         img = make_image(cfg, b, device)
         cond[b] = img["cond"]
         if uncond is not None:
             uncond[b] = img["uncond"]
         draft[b] = img["draft_lo"]
-        tok[b] = draw_draft_tokens(cfg, b, img["draft_lo"])
         del img
     nn = None
     if cfg.pool_k > 1:

@@ -11,7 +11,34 @@ import oracle as orc
 from paper_2601_05149_b200 import binding, synth
 
 
-build_batch = synth.build_batch
+_sampler_ctx = None
+
+
+def build_batch(cfg, images=None, device="cuda"):
+    """Seeded logits on the device plus the drafter's tokens.  The tokens of `images` (default: all)
+    are drawn by the ORACLE's sampler on the host, so that what the oracle is later given never came
+    from the CUDA path; the other images -- run on the device but not compared -- get theirs from the
+    library's sampler."""
+    global _sampler_ctx
+    batch = synth.build_batch(cfg, device)
+    images = list(range(cfg.B)) if images is None else sorted(set(images))
+    if len(images) < cfg.B:
+        if _sampler_ctx is None:
+            _sampler_ctx = binding.Context(0)
+        p = binding.params_from_config(cfg)
+        _sampler_ctx.ensure_workspace(p)
+        _sampler_ctx.mulo_sample_draft(p, batch["draft_lo"], batch["tok_lo"])
+        torch.cuda.synchronize()
+        _sampler_ctx.poll_device_status()
+
+    def one(b):
+        return orc.sample_draft_tokens(orc_params(cfg, b), synth.to_numpy_logits(batch["draft_lo"][b]))
+
+    orc.lib()
+    with cf.ThreadPoolExecutor(max_workers=min(16, max(1, len(images)))) as ex:
+        for b, tok in zip(images, ex.map(one, images)):
+            batch["tok_lo"][b] = torch.from_numpy(tok).to(device)
+    return batch
 
 
 def nn_numpy(batch):

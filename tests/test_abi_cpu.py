@@ -38,6 +38,16 @@ def test_status_strings(lib):
     assert len({binding.status_string(s) for s in range(6)}) == 6
 
 
+def test_timeout_bit_maps_to_an_error_status(lib):
+    """Host mapping of the device status word, on hand-set words (no kernel is made to time out)."""
+    report_bits = binding.DEV_ZERO_DRAFT_PROB | binding.DEV_BAD_TOKEN | binding.DEV_DENSE_FALLBACK
+    for word in (0, binding.DEV_DENSE_FALLBACK, report_bits):
+        assert binding.status_of_device_flags(word) == binding.OK
+    for word in (binding.DEV_TIMEOUT, binding.DEV_TIMEOUT | report_bits, 0xFFFFFFFF):
+        assert binding.status_of_device_flags(word) == binding.ERR_TIMEOUT
+    assert "timed out" in binding.status_string(binding.ERR_TIMEOUT)
+
+
 def _ws(p):
     n = C.c_size_t()
     return binding.lib().mulo_workspace_bytes(C.byref(p), C.byref(n)), n.value

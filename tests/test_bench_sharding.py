@@ -2,6 +2,7 @@
 reduction (gloo, world size 2) and the reference arm's launch contract under torchrun."""
 import json
 import os
+import socket
 import subprocess
 import sys
 
@@ -12,6 +13,13 @@ import torch.multiprocessing as mp
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 sys.path.insert(0, ROOT)
+
+
+def _free_port():
+    """A TCP port nobody listens on right now (asked of the kernel, so parallel test runs do not collide)."""
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
 
 
 def _worker(rank, world, port, out):
@@ -35,7 +43,7 @@ def _worker(rank, world, port, out):
 
 def test_two_ranks_shard_and_reduce(tmp_path):
     out = str(tmp_path / "r.json")
-    mp.spawn(_worker, args=(2, 29613, out), nprocs=2, join=True)
+    mp.spawn(_worker, args=(2, _free_port(), out), nprocs=2, join=True)
     r = json.load(open(out))
     assert r["slowest"] == 15.0                                 # max over ranks, not rank 0's own 10 ms
     (o0, s0, b0), (o1, s1, b1) = r["offsets"]
@@ -46,7 +54,7 @@ def test_two_ranks_shard_and_reduce(tmp_path):
 def test_reference_arm_under_torchrun():
     """Rank 0 alone runs the oracle and prints one JSON line; the other rank exits 0 without work."""
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
-           "--master-addr", "127.0.0.1", "--master-port", "29614", os.path.join(ROOT, "bench.py"),
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.join(ROOT, "bench.py"),
            "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0", "--workload", "C1"]
     p = subprocess.run(cmd, capture_output=True, text=True, timeout=600, cwd=ROOT)
     assert p.returncode == 0, p.stderr[-2000:]

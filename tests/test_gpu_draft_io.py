@@ -144,7 +144,7 @@ def test_downsample_random_tokens(ctx, r, alphabet):
 
 
 def test_downsample_undoes_replication_and_follows_a_round(ctx):
-    cfg = synth.RoundConfig("ds", B=3, H=16, W=24, V=512, r=2, dtype="bf16", top_k=64, sigma=1.0, radius=1,
+    cfg = synth.RoundConfig("ds", B=3, H=16, W=24, V=512, r=2, dtype="bf16", top_k=64, sigma=0.15, radius=1,
                             seed=320)
     batch = pu.build_batch(cfg)
     g = pu.gpu_round(ctx, cfg, batch)

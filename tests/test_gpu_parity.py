@@ -45,7 +45,7 @@ def _run(ctx, cfg, images=None, **over):
     dataclasses.replace(TINY, V=264, H=6, W=10, r=1, top_k=17, seed=106),          # ragged sizes
     dataclasses.replace(TINY, V=8, H=4, W=4, top_k=3, seed=107),                    # tiny vocabulary
     dataclasses.replace(TINY, H=12, W=36, r=3, radius=3, dtype="bf16", seed=108),   # two mask words per row
-    dataclasses.replace(TINY, V=2048, top_k=300, pool_k=128, pool_delta=0.1, dtype="bf16", seed=109),
+    dataclasses.replace(TINY, V=2048, top_k=300, pool_k=128, pool_delta=0.1, dtype="bf16", sigma=2.0, seed=109),
     dataclasses.replace(TINY, V=2048, top_k=0, pool_k=64, pool_delta=0.3, dtype="f32", seed=110),
 ], ids=lambda c: f"{c.dtype}-V{c.V}-k{c.top_k}-cfg{c.cfg_scale}-pool{c.pool_k}-{c.H}x{c.W}r{c.r}l{c.radius}")
 def test_round_small(ctx, cfg):
@@ -160,7 +160,7 @@ def test_config_C1(ctx):
 
 def test_config_C2(ctx):
     cfg = synth.CONFIGS["C2"]
-    batch = pu.build_batch(cfg)
+    batch = pu.build_batch(cfg, images=[0])
     g = pu.gpu_round(ctx, cfg, batch)
     o = pu.oracle_images(cfg, batch, [0])
     pu.check_round(cfg, g, o)
@@ -169,7 +169,7 @@ def test_config_C2(ctx):
 def test_config_C3_sampled_images(ctx):
     """Full-size batch on the GPU, first and last image against the oracle."""
     cfg = synth.CONFIGS["C3"]
-    batch = pu.build_batch(cfg)
+    batch = pu.build_batch(cfg, images=[0, cfg.B - 1])
     g = pu.gpu_round(ctx, cfg, batch)
     o = pu.oracle_images(cfg, batch, [0, cfg.B - 1])
     pu.check_round(cfg, g, o)
@@ -301,7 +301,7 @@ def test_config_C4_sampled_images(ctx):
     """The benchmark's workload in its launch configuration (B = 32 on the device),
     first and last image against the oracle, radii 1..3."""
     cfg = synth.CONFIGS["C4"]
-    batch = pu.build_batch(cfg)
+    batch = pu.build_batch(cfg, images=[0, cfg.B - 1])
     for radius in (3, 1, 2):
         c = dataclasses.replace(cfg, radius=radius)
         ctx.poll_fallback_counts()
@@ -331,7 +331,7 @@ def test_sweep_points_at_launch_size(ctx, cfg):
     """Points of the throughput sweep in the configuration the sweep times (B = 64 on the device): the
     first four images and the last against the oracle, no row redone by the general kernel."""
     assert cfg.B == 64
-    batch = pu.build_batch(cfg)
+    batch = pu.build_batch(cfg, images=[0, 1, 2, 3, cfg.B - 1])
     ctx.poll_fallback_counts()
     g = pu.gpu_round(ctx, cfg, batch)
     counts = ctx.poll_fallback_counts()      # rows redone, then by reason: list full, too few, above range, crowded bin
@@ -489,7 +489,7 @@ def test_round_is_bit_reproducible_at_launch_size(ctx):
     gives every output array bit for bit -- decisions depend on (seed, image, position, round) and the
     inputs only, not on how CTAs were scheduled."""
     cfg = synth.CONFIGS["C4"]
-    batch = pu.build_batch(cfg)
+    batch = pu.build_batch(cfg, images=[])      # nothing here goes to the oracle
     p = binding.params_from_config(cfg)
     ctx.ensure_workspace(p)
 

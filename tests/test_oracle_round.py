@@ -21,11 +21,13 @@ def _params(orc, cfg, image=0, **over):
 
 
 def _image(cfg, b=0):
+    import oracle
     img = synth.make_image(cfg, b)
-    tok = synth.draw_draft_tokens(cfg, b, img["draft_lo"])
+    draft = synth.to_numpy_logits(img["draft_lo"])
+    tok = oracle.sample_draft_tokens(_params(oracle, cfg, b), draft)
     return (synth.to_numpy_logits(img["cond"]),
             None if img["uncond"] is None else synth.to_numpy_logits(img["uncond"]),
-            synth.to_numpy_logits(img["draft_lo"]), tok.numpy())
+            draft, tok)
 
 
 SMALL = synth.RoundConfig("small", B=1, H=8, W=8, V=256, dtype="f32", sigma=0.7, radius=1, seed=11)
