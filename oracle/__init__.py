@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
             _lib.orc_expand.restype = C.c_int
             _lib.orc_islands.restype = C.c_int
             _lib.orc_island_schedule.restype = C.c_int
+            _lib.orc_redraw_loop.restype = C.c_int
     return _lib
 
 
@@ -203,6 +204,24 @@ def island_schedule(labels, window):
     step = np.zeros((H, W), np.int32)
     nfe = int(lib().orc_island_schedule(_ptr(labels), H, W, int(window), _ptr(step)))
     return step, nfe
+
+
+def redraw_loop(params, step, cond_steps, uncond_steps, tok, with_edge=False):
+    """The redraw of R_X, one target-model call per sequential step: ``cond_steps[s - 1]`` (and
+    ``uncond_steps[s - 1]``, or None) are the [H, W, V] logits of call s.  Returns the grid's tokens
+    after the redraw and the number of calls made."""
+    H, W = params.H, params.W
+    step = np.ascontiguousarray(step, np.int32)
+    n_steps = int(step.max()) if step.size else 0
+    assert len(cond_steps) >= n_steps
+    conds = [np.ascontiguousarray(c) for c in cond_steps[:n_steps]]
+    unconds = None if uncond_steps is None else [np.ascontiguousarray(u) for u in uncond_steps[:n_steps]]
+    arr = (C.c_void_p * max(1, n_steps))(*[c.ctypes.data for c in conds])
+    uarr = None if unconds is None else (C.c_void_p * max(1, n_steps))(*[u.ctypes.data for u in unconds])
+    out = np.array(tok, np.int32, copy=True).reshape(H, W)
+    edge = np.zeros((H, W), np.uint8)
+    calls = int(lib().orc_redraw_loop(C.byref(params), _ptr(step), n_steps, arr, uarr, _ptr(out), _ptr(edge)))
+    return (out, calls, edge) if with_edge else (out, calls)
 
 
 def position_distributions(params, cond_row, uncond_row, draft_row, tok, nn=None):

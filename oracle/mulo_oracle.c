@@ -645,6 +645,48 @@ void orc_sample_draft_tokens(const orc_params* P, const void* draft_lo, int32_t*
   free(q);
 }
 
+/* The redraw of R_X executed step by step (Sec. 3.4, Algorithm 1 Step 6).  The target model
+ * is called once per sequential step s = 1 .. n_steps of the schedule; a call yields logits for
+ * the whole grid given the tokens decoded so far, and the positions with step(t) == s take their
+ * token from them: one draw from the target distribution (CFG, temperature, top-k as in the round)
+ * by inverse CDF in ascending token id.  Here the model calls are an input: cond_steps[s - 1]
+ * (and uncond_steps[s - 1], or uncond_steps == NULL) is the [H*W, V] logit tensor of call s.
+ * Reading: the uniform of position t at step s is word 0 of the Philox stream with counter
+ * (t, image, round, 1 + s) -- tag 0 holds the round's own uniforms and tag 1 the drafter's draw,
+ * so the redraw's numbers are new ones and a position redrawn in two different rounds or steps
+ * never reuses a uniform (the paper does not say how the redraw is seeded).
+ *   step [H*W]  the schedule (0 outside R_X);   tok [H*W] in/out: positions outside R_X keep
+ *   their token;   edge [H*W] out, may be NULL: 1 where the uniform lies within 1e-6 of an edge
+ *   of the chosen CDF bin.
+ * Returns the number of target-model calls made (the NFE of the redraw): n_steps. */
+int orc_redraw_loop(const orc_params* P, const int32_t* step, int n_steps, const void* const* cond_steps,
+                    const void* const* uncond_steps, int32_t* tok, uint8_t* edge) {
+  const int V = P->V, N = P->H * P->W;
+  const size_t esz = P->dtype == ORC_BF16 ? 2 : 4;
+  float* z = (float*)malloc((size_t)V * sizeof(float));
+  double* p = (double*)malloc((size_t)V * sizeof(double));
+  int calls = 0;
+  if (edge) memset(edge, 0, (size_t)N);
+  for (int s = 1; s <= n_steps; ++s) {
+    const char* cond = (const char*)cond_steps[s - 1];
+    const char* uncond = uncond_steps ? (const char*)uncond_steps[s - 1] : NULL;
+    ++calls;
+    for (int t = 0; t < N; ++t) {
+      if (step[t] != s) continue;
+      double m, Z, u[3], gap;
+      orc_preprocess_row(cond + (size_t)t * V * esz, uncond ? uncond + (size_t)t * V * esz : NULL, P->dtype, V,
+                         P->cfg_scale, P->temperature, z);
+      orc_softmax_masked(z, V, orc_topk_threshold(z, V, P->top_k), p, &m, &Z);
+      orc_position_uniforms(P->seed, P->image, (uint32_t)t, P->round, 1u + (uint32_t)s, u);
+      tok[t] = orc_inverse_cdf(p, V, u[0], NULL, &gap);
+      if (edge) edge[t] = gap < 1e-6;
+    }
+  }
+  free(z);
+  free(p);
+  return calls;
+}
+
 /* Step 7 stand-in.  The paper's D_r is a trained network; the stand-in keeps the
  * one property the round relies on, D_r(U_r(y)) = y for the replicating U_r:
  * y[a][c] is the token that occurs most often among the r x r tokens
