@@ -286,8 +286,9 @@ def run_ours(args, cfg):
         peak, peak_src = 6650.0, "fallback (6.65 TB/s)"
     row_avg_ms = row_ms / max(1, row_n)
     achieved = alg_bytes / (row_avg_ms * 1e-3) / 1e9
-    which = ctx.round_kernel(p)
-    kernel = {"lane": "k_round_lane (+ k_verify_failed for rows that left the fast path)",
+    which = ctx.round_kernel(p, cfg.has_uncond)
+    kernel = {"full": "k_round_full",
+              "lane": "k_round_lane (+ k_verify_failed for rows that left the fast path)",
               "stream": "k_round_stream (+ k_verify_failed for rows that left the fast path)",
               "general": "k_verify_rows"}[which]
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,

@@ -147,8 +147,13 @@ mulo_status mulo_status_of_device_flags(uint32_t flags);
 mulo_status mulo_poll_fallback_counts(mulo_ctx* ctx, void* stream, uint32_t counts[5]);
 /* Number of kernels this context has launched so far. */
 mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
-/* mulo_round picks between three row kernels, mulo_sample_draft between the last two.  All
+/* mulo_round picks between four row kernels, mulo_sample_draft between the last two.  All
  * compute the same function; a row a fast kernel cannot handle is redone by the general routines.
+ *   MULO_KERNEL_FULL     top-k off (the paper's default sampling), V a multiple of 2048 (bf16) or
+ *                        1024 (fp32), the rows of one position within a CTA's shared memory (e.g.
+ *                        V <= 16384 in bf16 with classifier-free guidance): rows are made resident
+ *                        in shared memory and every entry is exponentiated once; with Eq. 5 and
+ *                        redraws from the target distribution the draft logits are not read;
  *   MULO_KERNEL_LANE     top-k on, pooling off, V a multiple of 4096 (bf16) or 2048 (fp32) and
  *                        at most 16384: every thread of a CTA owns a contiguous range of the
  *                        vocabulary, rows are streamed once through per-warp shared-memory rings;
@@ -156,11 +161,13 @@ mulo_status mulo_kernel_launches(const mulo_ctx* ctx, uint64_t* count);
  *                        streamed once in chunks, candidates compacted per segment;
  *   MULO_KERNEL_GENERAL  everything else (top-k off, tiny vocabularies): one CTA per row, the
  *                        row read several times (from L2 after the first).
- * mulo_round_kernel reports the choice for these parameters on this context (host arithmetic
- * only; nothing is launched).  mulo_set_general_path_only(on != 0) makes the context always use
+ * mulo_round_kernel reports the choice for these parameters (and with or without an unconditional
+ * tensor) on this context (host arithmetic only; nothing is launched).  mulo_set_general_path_only(on != 0) makes the context always use
  * the general kernel (for testing and comparison). */
-typedef enum { MULO_KERNEL_GENERAL = 0, MULO_KERNEL_STREAM = 1, MULO_KERNEL_LANE = 2 } mulo_kernel;
-mulo_status mulo_round_kernel(const mulo_ctx* ctx, const mulo_params* p, int* kernel);
+typedef enum {
+  MULO_KERNEL_GENERAL = 0, MULO_KERNEL_STREAM = 1, MULO_KERNEL_LANE = 2, MULO_KERNEL_FULL = 3
+} mulo_kernel;
+mulo_status mulo_round_kernel(const mulo_ctx* ctx, const mulo_params* p, int has_uncond, int* kernel);
 mulo_status mulo_set_general_path_only(mulo_ctx* ctx, int on);
 /* Optional device timing of the fused row kernel (the launch that reads the logits):
  * mulo_set_timing prepares CUDA event pairs for up to max_launches (<= 4096) calls of
@@ -278,10 +285,43 @@ mulo_status mulo_resample(mulo_ctx* ctx, const mulo_params* p, const void* tgt_c
                           const uint16_t* nn, const uint32_t* reject_bits,
                           const uint32_t* expand_bits, int32_t* out_tok, void* stream);
 
+/* ---- the redraw of R_X, step by step (Sec. 3.4, Algorithm 1 Step 6) ------------------------ */
+
+/* Sorts the positions of R_X by their step of the schedule (mulo_island_schedule), on the device:
+ *   step         [B, H, W]             in   1-based step of each position, 0 outside R_X
+ *   max_step                                an upper bound of the steps present, 1 <= max_step <= H W
+ *                                           (positions with a larger step are left out)
+ *   pos_list     [B H W]               out  position indices b H W + t, the positions of step 1 first,
+ *                                           then step 2, ...; order within a step unspecified
+ *   step_offsets [2 (max_step + 2)]    out  entry s (1 <= s <= max_step) = where step s starts in
+ *                                           pos_list, entry max_step + 1 = where the last step ends;
+ *                                           the second half of the array is scratch
+ * Three small launches, no host round-trip.  Needs no workspace. */
+mulo_status mulo_redraw_plan(mulo_ctx* ctx, const mulo_params* p, const int32_t* step, int32_t max_step,
+                             int32_t* pos_list, int32_t* step_offsets, void* stream);
+/* One sequential step s of the redraw: every position of step s takes a new token, drawn from the
+ * target distribution p(. | the given logits) -- CFG mix, temperature and top-k as in the round,
+ * inverse CDF in ascending token id.  The logits stand for the target model's call number s (the
+ * model is not part of this library): tgt_cond / tgt_uncond are [B, H, W, V] tensors of which only
+ * the rows of this step's positions are read.  The uniform of position t is word 0 of Philox4x32-10
+ * at counter (t, image_offset + b, round, 1 + s): a stream of its own beside the round's (tag 0) and
+ * the drafter's (tag 1); the paper does not say how the redraw is seeded.  One launch whose grid
+ * does not depend on how many positions the step has (their number stays on the device).
+ *   s, max_step                     1 <= s <= max_step, max_step as given to mulo_redraw_plan
+ *   pos_list, step_offsets     in   from mulo_redraw_plan
+ *   out_tok [B, H, W]          in/out  int32; only this step's positions are written           */
+mulo_status mulo_redraw_step(mulo_ctx* ctx, const mulo_params* p, int32_t s, int32_t max_step,
+                             const int32_t* pos_list, const int32_t* step_offsets, const void* tgt_cond,
+                             const void* tgt_uncond, int32_t* out_tok, void* stream);
+
 /* ---- the fused round ------------------------------------------------------------------- */
 
 /* The four stages in one pass: every logit row is read from HBM once.  Results are those
- * of mulo_upsample_pool -> mulo_verify -> mulo_local_reject_expand -> mulo_resample.
+ * of mulo_upsample_pool -> mulo_verify -> mulo_local_reject_expand -> mulo_resample, with one
+ * exception: with MULO_ACCEPT_THRESHOLD and MULO_RESAMPLE_TARGET_ALL (Eq. 5 as printed, every
+ * redraw from the target distribution) neither the decision nor any draw depends on the draft
+ * distribution, so q_tok, if given, is filled with zeros, and where the resident-row kernel
+ * runs (MULO_KERNEL_FULL) draft_logits_lo is not read at all (it must still be a valid pointer).
  *   p_tok, q_tok, accept_prob may be NULL (skipped).  Needs the workspace. */
 mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond,
                        const void* tgt_uncond, const void* draft_logits_lo,

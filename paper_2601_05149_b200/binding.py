@@ -26,6 +26,7 @@ EXPORTS = (
     "mulo_kernel_launches",
     "mulo_set_timing", "mulo_read_timing", "mulo_set_general_path_only", "mulo_round_kernel",
     "mulo_upsample_pool", "mulo_verify", "mulo_local_reject_expand", "mulo_islands", "mulo_island_schedule", "mulo_sample_draft", "mulo_downsample", "mulo_resample",
+    "mulo_redraw_plan", "mulo_redraw_step",
     "mulo_round", "mulo_round_host_arena_bytes", "mulo_round_host", "mulo_round_static",
 )
 
@@ -198,11 +199,11 @@ class Context:
         _check(lib().mulo_kernel_launches(self._ctx, C.byref(n)), "mulo_kernel_launches")
         return n.value
 
-    def round_kernel(self, p: "MuloParams") -> str:
-        """The row kernel ``mulo_round`` launches for these parameters: "lane", "stream" or "general"."""
+    def round_kernel(self, p: "MuloParams", has_uncond: bool) -> str:
+        """The row kernel ``mulo_round`` launches for these parameters: "full", "lane", "stream" or "general"."""
         k = C.c_int()
-        _check(lib().mulo_round_kernel(self._ctx, C.byref(p), C.byref(k)), "mulo_round_kernel")
-        return ("general", "stream", "lane")[k.value]
+        _check(lib().mulo_round_kernel(self._ctx, C.byref(p), int(has_uncond), C.byref(k)), "mulo_round_kernel")
+        return ("general", "stream", "lane", "full")[k.value]
 
     def set_general_path_only(self, on: bool):
         _check(lib().mulo_set_general_path_only(self._ctx, int(bool(on))), "mulo_set_general_path_only")
@@ -266,6 +267,15 @@ class Context:
                                    _dev(draft_logits_lo), _dev(draft_stats_lo), _dev(draft_tok_hi),
                                    _dev(nn), _dev(reject_bits), _dev(expand_bits), _dev(out_tok),
                                    _stream(stream)), "mulo_resample")
+
+    def mulo_redraw_plan(self, p, step, max_step, pos_list, step_offsets, stream=None):
+        _check(lib().mulo_redraw_plan(self._ctx, C.byref(p), _dev(step), int(max_step), _dev(pos_list),
+                                      _dev(step_offsets), _stream(stream)), "mulo_redraw_plan")
+
+    def mulo_redraw_step(self, p, s, max_step, pos_list, step_offsets, tgt_cond, tgt_uncond, out_tok, stream=None):
+        _check(lib().mulo_redraw_step(self._ctx, C.byref(p), int(s), int(max_step), _dev(pos_list),
+                                      _dev(step_offsets), _dev(tgt_cond), _dev(tgt_uncond), _dev(out_tok),
+                                      _stream(stream)), "mulo_redraw_step")
 
     def mulo_round(self, p, tgt_cond, tgt_uncond, draft_logits_lo, draft_tok_lo, nn, out_tok,
                    reject_bits, expand_bits, p_tok=None, q_tok=None, accept_prob=None, n_reject=None,

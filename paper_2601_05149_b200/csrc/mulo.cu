@@ -12,6 +12,7 @@
 #include "mulo_dense.cuh"
 #include "mulo_islands.cuh"
 #include "mulo_lane.cuh"
+#include "mulo_full.cuh"
 #include "mulo_stream.cuh"
 
 using namespace mulo;
@@ -132,6 +133,97 @@ __global__ void __launch_bounds__(kThreads) k_sample_failed(RowKernelArgs a, con
   for (size_t idx = blockIdx.x; idx < n; idx += gridDim.x) {
     const size_t cell = (size_t)fail_list[idx];
     if (cell < total) sample_cell(a, (int)cell, bs);
+    __syncthreads();
+  }
+}
+
+// ---- the redraw of R_X, one launch per sequential step (Sec. 3.4, Algorithm 1 Step 6)
+// Plan: the positions sorted by their step -- count, scan, fill.  offsets[s] is where step s starts in
+// pos_list (s = 1 .. max_step, offsets[max_step + 1] the end); the cursors live behind the offsets.
+constexpr int kScanThreads = 1024;
+
+__global__ void __launch_bounds__(256) k_redraw_count(const int32_t* __restrict__ step, int n, int max_step,
+                                                      int32_t* cursor) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int s = step[i];
+    if (s >= 1 && s <= max_step) atomicAdd(&cursor[s], 1);
+  }
+}
+
+__global__ void __launch_bounds__(kScanThreads) k_redraw_scan(int max_step, int32_t* offsets, int32_t* cursor) {
+  __shared__ int warp_tot[kScanThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = max_step + 1;                       // entries 0 .. max_step (entry 0 counts nothing)
+  const int per = (n + kScanThreads - 1) / kScanThreads;
+  const int beg = min(n, tid * per), end = min(n, beg + per);
+  int mine = 0;
+  for (int i = beg; i < end; ++i) mine += i == 0 ? 0 : cursor[i];
+  int inc = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(kFull, inc, o);
+    if (lane >= o) inc += v;
+  }
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  int pre = 0;
+  for (int w = 0; w < warp; ++w) pre += warp_tot[w];
+  int run = pre + inc - mine;                        // positions with a step below this thread's first
+  for (int i = beg; i < end; ++i) {
+    const int c = i == 0 ? 0 : cursor[i];
+    offsets[i] = run;
+    cursor[i] = run;
+    run += c;
+  }
+  if (tid == kScanThreads - 1) offsets[max_step + 1] = pre + inc;   // (the last thread's inclusive sum: the total)
+}
+
+__global__ void __launch_bounds__(256) k_redraw_fill(const int32_t* __restrict__ step, int n, int max_step,
+                                                     int32_t* cursor, int32_t* pos_list) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int s = step[i];
+    if (s >= 1 && s <= max_step) pos_list[atomicAdd(&cursor[s], 1)] = i;
+  }
+}
+
+struct RedrawArgs {
+  DevParams P;
+  const char* cond;
+  const char* uncond;
+  const int32_t* pos_list;
+  const int32_t* offsets;
+  int32_t* out_tok;
+  int s;
+};
+
+// One step: every position of the step's slice of the list draws its token from the target
+// distribution of the given logits; uniform = word 0 of Philox at (t, image, round, 1 + s).
+__global__ void __launch_bounds__(kThreads) k_redraw_step(RedrawArgs a) {
+  __shared__ BlockScratch bs;
+  const DevParams& P = a.P;
+  const int beg = a.offsets[a.s], end = a.offsets[a.s + 1];
+  const size_t N = (size_t)P.H * P.W, total = (size_t)P.B * N;
+  const size_t bytes = (size_t)P.V * (P.bf16 ? 2 : 4);
+  for (int i = beg + (int)blockIdx.x; i < end; i += (int)gridDim.x) {
+    const size_t g = (size_t)a.pos_list[i];
+    if (g < total) {   // block-uniform
+      const uint32_t b = (uint32_t)(g / N), t = (uint32_t)(g - (size_t)b * N);
+      RowSrc tr;
+      tr.cond = a.cond + g * bytes;
+      tr.uncond = a.uncond ? a.uncond + g * bytes : nullptr;
+      tr.s = P.cfg_scale;
+      tr.invT = P.invT;
+      tr.V = P.V;
+      tr.bf16 = P.bf16;
+      RowStats sp;
+      dense_row_stats(tr, P.top_k, bs, sp.theta, sp.m, sp.Z);
+      __syncthreads();
+      const float invZ = (float)(1.0 / sp.Z);
+      const uint4 rnd = philox4x32_10(make_uint4(t, b + P.image_offset, P.round, 1u + (uint32_t)a.s),
+                                      make_uint2(P.seed_lo, P.seed_hi));
+      const int tok = dense_draw(tr, tr, sp, sp, invZ, invZ, 0.0f, -1, 0.0, nullptr, uniform24(rnd.x), bs);
+      if (threadIdx.x == 0) a.out_tok[g] = tok;
+    }
     __syncthreads();
   }
 }
@@ -875,6 +967,50 @@ static size_t plan_lane(const mulo_ctx* ctx, const DevParams& d, LaneArgs* s) {
   return dyn;
 }
 
+// ---- rows without a top-k cut: the resident-row kernel ------------------------------------
+// Eligible: top-k off, V = 256 * W with W a multiple of the ids in 16 bytes, and the rows of one
+// position (draft row if q is needed, conditional, unconditional) within a CTA's shared memory.
+static bool round_needs_q(const DevParams& d) {
+  return !(d.accept_mode == MULO_ACCEPT_THRESHOLD && d.resample_mode == MULO_RESAMPLE_TARGET_ALL);
+}
+
+static size_t plan_full(const mulo_ctx* ctx, const DevParams& d, bool has_u, FullArgs* s) {
+  if (d.top_k > 0 && d.top_k < d.V) return 0;
+  const int esz = d.bf16 ? 2 : 4, n = 16 / esz;
+  if (d.V % (kFThreads * n) != 0) return 0;
+  const int need_q = round_needs_q(d) ? 1 : 0;
+  const size_t rows = (size_t)need_q + 1 + (has_u ? 1 : 0);
+  const size_t dyn = rows * (size_t)d.V * esz + (size_t)d.V / 8 + (size_t)kFThreads * 8;
+  if (dyn + sizeof(FullSmem) + 1024 > (size_t)ctx->smem_optin) return 0;
+  s->W = d.V / kFThreads;
+  s->need_q = need_q;
+  return dyn;
+}
+
+template <bool BF16, bool HAS_U>
+static bool launch_full_t(const mulo_ctx* ctx, const FullArgs& s, size_t dyn, cudaStream_t st) {
+  auto kern = k_round_full<BF16, HAS_U>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kFThreads, dyn) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return false;
+  }
+  int grid = ctx->sm_count * per_sm;
+  if (grid > s.n_parents) grid = s.n_parents;
+  kern<<<grid, kFThreads, dyn, st>>>(s);
+  return true;
+}
+
+static bool launch_full(const mulo_ctx* ctx, const FullArgs& s, size_t dyn, cudaStream_t st) {
+  const bool hu = s.uncond != nullptr;
+  if (s.P.bf16) return hu ? launch_full_t<true, true>(ctx, s, dyn, st) : launch_full_t<true, false>(ctx, s, dyn, st);
+  return hu ? launch_full_t<false, true>(ctx, s, dyn, st) : launch_full_t<false, false>(ctx, s, dyn, st);
+}
+
 template <bool BF16, bool HAS_U>
 static bool launch_lane_t(const mulo_ctx* ctx, const LaneArgs& s, const CUtensorMap& tc, const CUtensorMap& tu,
                           const CUtensorMap& tq, size_t dyn, cudaStream_t st) {
@@ -969,6 +1105,51 @@ mulo_status mulo_island_schedule(mulo_ctx* ctx, const mulo_params* p, const int3
     return MULO_ERR_CUDA;
   }
   k_island_schedule<<<p->B, kScheduleThreads, smem, (cudaStream_t)stream>>>(a);
+  return launched(ctx, 1);
+}
+
+mulo_status mulo_redraw_plan(mulo_ctx* ctx, const mulo_params* p, const int32_t* step, int32_t max_step,
+                             int32_t* pos_list, int32_t* step_offsets, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!step || !pos_list || !step_offsets || max_step < 1) return MULO_ERR_INVALID_ARG;
+  if ((size_t)max_step > (size_t)p->H * p->W) return MULO_ERR_INVALID_ARG;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int n = p->B * p->H * p->W;
+  int32_t* cursor = step_offsets + max_step + 2;
+  if (cudaMemsetAsync(step_offsets, 0, sizeof(int32_t) * 2 * ((size_t)max_step + 2), st) != cudaSuccess) return MULO_ERR_CUDA;
+  if (n == 0) return MULO_OK;
+  const int blocks = (n + 255) / 256 < 4 * ctx->sm_count ? (n + 255) / 256 : 4 * ctx->sm_count;
+  k_redraw_count<<<blocks, 256, 0, st>>>(step, n, max_step, cursor);
+  k_redraw_scan<<<1, kScanThreads, 0, st>>>(max_step, step_offsets, cursor);
+  k_redraw_fill<<<blocks, 256, 0, st>>>(step, n, max_step, cursor, pos_list);
+  return launched(ctx, 3);
+}
+
+mulo_status mulo_redraw_step(mulo_ctx* ctx, const mulo_params* p, int32_t s_index, int32_t max_step,
+                             const int32_t* pos_list, const int32_t* step_offsets, const void* tgt_cond,
+                             const void* tgt_uncond, int32_t* out_tok, void* stream) {
+  if (!ctx) return MULO_ERR_INVALID_ARG;
+  mulo_status s = validate(p);
+  if (s != MULO_OK) return s;
+  if (!pos_list || !step_offsets || !tgt_cond || !out_tok || !aligned16(tgt_cond) || !aligned16(tgt_uncond))
+    return MULO_ERR_INVALID_ARG;
+  if (s_index < 1 || s_index > max_step) return MULO_ERR_INVALID_ARG;
+  if (p->B == 0) return MULO_OK;
+  if ((s = on_context_device(ctx)) != MULO_OK) return s;
+  RedrawArgs a;
+  memset(&a, 0, sizeof a);
+  a.P = to_dev(p);
+  a.cond = (const char*)tgt_cond;
+  a.uncond = (const char*)tgt_uncond;
+  a.pos_list = pos_list;
+  a.offsets = step_offsets;
+  a.out_tok = out_tok;
+  a.s = s_index;
+  // the step's positions are counted on the device: a fixed grid strides over them
+  k_redraw_step<<<2 * ctx->sm_count, kThreads, 0, (cudaStream_t)stream>>>(a);
   return launched(ctx, 1);
 }
 
@@ -1176,9 +1357,31 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   const bool timed = ctx->ev_used + 2 <= ctx->ev.size();
   if (timed) cudaEventRecord(ctx->ev[ctx->ev_used], st);
   bool fast = false;
+  int fast_launches = 2;   // a fast kernel and the one that redoes the rows it left
+  // Eq. 5 with every redraw from the target distribution never looks at q: no kernel reports it
+  // (the resident-row kernel does not even read the draft logits), the output is zero-filled
+  if (!round_needs_q(a.P) && q_tok) {
+    if (cudaMemsetAsync(q_tok, 0, sizeof(float) * (size_t)p->B * p->H * p->W, st) != cudaSuccess) return MULO_ERR_CUDA;
+    a.q_tok = nullptr;
+    q_tok = nullptr;
+  }
+  FullArgs fa;
+  memset(&fa, 0, sizeof fa);
+  const size_t fdyn = ctx->force_dense ? 0 : plan_full(ctx, a.P, tgt_uncond != nullptr, &fa);
+  if (fdyn) {
+    fa.P = a.P;
+    fa.cond = a.cond; fa.uncond = a.uncond; fa.draft = a.draft; fa.draft_tok_lo = draft_tok_lo;
+    fa.nn = a.nn;
+    fa.p_tok = p_tok; fa.q_tok = q_tok; fa.accept_prob = accept_prob;
+    fa.flags = w.flags; fa.cand_res = w.cand_res; fa.cand_tgt = w.cand_tgt;
+    fa.dev_status = w.status;
+    fa.n_parents = p->B * a.P.h * a.P.w;
+    fast = launch_full(ctx, fa, fdyn, st);
+    if (fast) fast_launches = 1;
+  }
   LaneArgs la;
   memset(&la, 0, sizeof la);
-  const size_t ldyn = (ctx->force_dense || ctx->no_lane) ? 0 : plan_lane(ctx, a.P, &la);
+  const size_t ldyn = (ctx->force_dense || ctx->no_lane || fast) ? 0 : plan_lane(ctx, a.P, &la);
   if (ldyn) {
     la.P = a.P;
     la.cond = a.cond; la.uncond = a.uncond; la.draft = a.draft; la.draft_tok_lo = draft_tok_lo;
@@ -1222,10 +1425,10 @@ mulo_status mulo_round(mulo_ctx* ctx, const mulo_params* p, const void* tgt_cond
   m.cand_res = w.cand_res; m.cand_tgt = w.cand_tgt;
   m.draft_tok_lo = draft_tok_lo; m.out_tok = out_tok;
   k_mask<2><<<p->B, kMaskThreads, mask_smem(p), st>>>(m);
-  return launched(ctx, fast ? 3 : 2);
+  return launched(ctx, fast ? 1 + fast_launches : 2);
 }
 
-mulo_status mulo_round_kernel(const mulo_ctx* ctx, const mulo_params* p, int* kernel) {
+mulo_status mulo_round_kernel(const mulo_ctx* ctx, const mulo_params* p, int has_uncond, int* kernel) {
   if (!ctx || !kernel) return MULO_ERR_INVALID_ARG;
   const mulo_status s = validate(p);
   if (s != MULO_OK) return s;
@@ -1236,7 +1439,10 @@ mulo_status mulo_round_kernel(const mulo_ctx* ctx, const mulo_params* p, int* ke
   memset(&sa, 0, sizeof sa);
   *kernel = MULO_KERNEL_GENERAL;
   if (ctx->force_dense) return MULO_OK;
-  if (!ctx->no_lane && plan_lane(ctx, d, &la)) *kernel = MULO_KERNEL_LANE;
+  FullArgs fa;
+  memset(&fa, 0, sizeof fa);
+  if (plan_full(ctx, d, has_uncond != 0, &fa)) *kernel = MULO_KERNEL_FULL;
+  else if (!ctx->no_lane && plan_lane(ctx, d, &la)) *kernel = MULO_KERNEL_LANE;
   else if (plan_stream(ctx, d, &sa)) *kernel = MULO_KERNEL_STREAM;
   return MULO_OK;
 }

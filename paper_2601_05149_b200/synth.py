@@ -1,7 +1,6 @@
 """Seeded synthetic inputs for the MuLo-SD draft-and-verify round.
 
-This module only MAKES INPUTS (logit tensors, draft tokens, codebook neighbour
-lists).  It holds none of the round's arithmetic and is the one module that both
+This module only MAKES INPUTS (logit tensors, codebook neighbour lists).  It holds none of the round's arithmetic and is the one module that both
 the CUDA tests/benchmark and the CPU oracle's tests draw their data from.
 
 Recipe (per image ``b`` of a config with seed ``s``; generator seed
@@ -15,7 +14,8 @@ Recipe (per image ``b`` of a config with seed ``s``; generator seed
    rounded;
 4. draft tokens ``[h, w]``: one draw per low-res cell from the draft distribution
    (temperature and top-k applied) -- the drafter's own sampling step, which the
-   round takes as an input;
+   round takes as an input.  They are NOT drawn here: callers use the library's
+   ``mulo_sample_draft`` or, where the tokens feed the oracle, the oracle's sampler;
 5. with probability pooling: a synthetic codebook ``E ~ N(0,1)^{V x 8}`` and, per
    token, the ``k`` nearest codebook entries by L2 distance (self first, ties to
    the lower id) as ``uint16``.
@@ -79,7 +79,10 @@ class RoundConfig:
         row(s), the parent's draft row shared by r*r children, the neighbour list
         when pooling is on, and the per-position outputs."""
         v = self.V * self.elem_size
-        return v * (2 if self.has_uncond else 1) + v / (self.r * self.r) + \
+        # Eq. 5 with every redraw from the target distribution never looks at the draft row
+        # (accept_mode 1 = threshold rule, resample_mode 2 = target for all)
+        draft = 0.0 if (self.accept_mode == 1 and self.resample_mode == 2) else v / (self.r * self.r)
+        return v * (2 if self.has_uncond else 1) + draft + \
             (2 * self.pool_k if self.pool_k > 1 else 0) + 24
 
 
@@ -92,6 +95,11 @@ CONFIGS = {
                       radius=1, seed=2),
     "C4": RoundConfig("C4", B=32, H=64, W=64, V=16384, sigma=1.0, cfg_scale=3.0, top_k=2000,
                       radius=3, seed=3),
+    # C4's shapes under the paper's default sampling: no top-k cut, CFG 4.0, probability pooling over
+    # the k = 1000 nearest codebook entries with delta = 0.1, the relaxed rule of Eq. 5 with tau = 1e-4,
+    # every redraw from the target distribution, l = 3
+    "P4": RoundConfig("P4", B=32, H=64, W=64, V=16384, sigma=1.0, cfg_scale=4.0, top_k=0, pool_k=1000,
+                      pool_delta=0.1, radius=3, accept_mode=1, tau=1e-4, resample_mode=2, seed=5),
 }
 
 

@@ -31,14 +31,22 @@ def build_batch(cfg, images=None, device="cuda"):
         torch.cuda.synchronize()
         _sampler_ctx.poll_device_status()
 
+    redraw_tokens(cfg, batch, images)
+    return batch
+
+
+def redraw_tokens(cfg, batch, images=None):
+    """The drafter's tokens of `images` (default: all) from the batch's current draft logits, by the
+    oracle's sampler (after a test has transformed the logits, so that q(x~) > 0 again)."""
+    images = list(range(cfg.B)) if images is None else images
+
     def one(b):
         return orc.sample_draft_tokens(orc_params(cfg, b), synth.to_numpy_logits(batch["draft_lo"][b]))
 
     orc.lib()
     with cf.ThreadPoolExecutor(max_workers=min(16, max(1, len(images)))) as ex:
         for b, tok in zip(images, ex.map(one, images)):
-            batch["tok_lo"][b] = torch.from_numpy(tok).to(device)
-    return batch
+            batch["tok_lo"][b] = torch.from_numpy(tok).to(batch["tok_lo"].device)
 
 
 def nn_numpy(batch):
@@ -186,7 +194,11 @@ def compare_image(cfg, g, b, o, prob_rtol):
         f"image {b}: token differs at unflagged positions {np.argwhere(bad_tok & ~draw_edge)[:5]}"
     assert int(g["n_reject"][b]) == int(rej_g.sum()) and int(g["n_expand"][b]) == int(g["expand"][b].sum())
     if "p_tok" in g:
-        for k in ("p_tok", "q_tok", "accept_prob"):
+        # Eq. 5 with every redraw from the target distribution: q is never looked at and reported as zero
+        no_q = cfg.accept_mode == binding.ACCEPT_THRESHOLD and cfg.resample_mode == binding.RESAMPLE_TARGET_ALL
+        if no_q:
+            assert np.all(g["q_tok"][b] == 0)
+        for k in ("p_tok", "accept_prob") if no_q else ("p_tok", "q_tok", "accept_prob"):
             want = o[k]
             sel = want >= 1e-30
             if k != "q_tok":
@@ -220,5 +232,12 @@ def check_round(cfg, g, oracle_out, prob_rtol=None):
     FRACTIONS.append((cfg.name, total, flagged / total, excused / total))
     print(f"[parity] {cfg.name}: {total} positions, flagged_fraction {flagged / total:.3e}, "
           f"excused_fraction {excused / total:.3e}")
-    assert excused <= max(1, int(1e-4 * total)) or excused / total < 1e-4, (excused, total)
+    # The flagged positions are a slice of the unit interval that grows with the number n of active
+    # tokens (2e-6 * n: 0.4 % at top-k 2000, 3.3 % for 16384 tokens without a cut).  A flagged draw comes
+    # out differently only if its uniform falls between the oracle's CDF edge and the GPU's, whose fp32
+    # weights (each within about 1e-7 relative) move an edge by a few 1e-8 of normalised mass: a few
+    # per cent of the 1e-6 band.  So the budget is 1e-4 of all positions, or 3 % of the flagged ones
+    # where that is more (only rows without a top-k cut get there).
+    allowed = max(1, int(1e-4 * total), int(0.03 * flagged))
+    assert excused <= allowed or excused / total < 1e-4, (excused, flagged, total)
     return excused, flagged

@@ -399,10 +399,7 @@ def test_pooling_on_the_streaming_path(ctx, scale, pool_k, delta):
     batch = pu.build_batch(cfg)
     for k in ("cond", "uncond", "draft_lo"):
         batch[k] = (batch[k].float() * scale).to(batch[k].dtype).contiguous()
-    p = binding.params_from_config(cfg)
-    ctx.ensure_workspace(p)
-    ctx.mulo_sample_draft(p, batch["draft_lo"], batch["tok_lo"])     # draft tokens with q > 0 under the new logits
-    torch.cuda.synchronize()
+    pu.redraw_tokens(cfg, batch)                                      # draft tokens with q > 0 under the new logits
     n0 = ctx.kernel_launches()
     g = pu.gpu_round(ctx, cfg, batch)
     assert ctx.kernel_launches() - n0 == 3                            # streaming kernel, its list, the mask kernel
@@ -510,3 +507,59 @@ def test_round_is_bit_reproducible_at_launch_size(ctx):
         assert first[k].tobytes() == second[k].tobytes(), k
         assert first[k].tobytes() == third[k].tobytes(), k
     assert ctx.poll_device_status() & ~binding.DEV_DENSE_FALLBACK == 0
+
+
+# ------------------------------------------------------------------ rows without a top-k cut
+
+@pytest.mark.parametrize("tau", [1e-3, 1e-4, 5e-5, 1e-5])
+@pytest.mark.parametrize("accept_mode", [binding.ACCEPT_THRESHOLD, binding.ACCEPT_RATIO], ids=["eq5", "eq1"])
+def test_paper_default_sampling(ctx, tau, accept_mode):
+    """The paper's default sampling on the benchmark's shapes: no top-k cut, CFG 4.0, pooling over the
+    1000 nearest codebook entries with delta = 0.1, l = 3; Eq. 5 (redraws from the target distribution)
+    for four thresholds, and Eq. 1 with the same pooling (residual redraws at rejections).  64x64 at
+    B = 2, both images against the oracle; the rows run on the resident-row kernel."""
+    if accept_mode == binding.ACCEPT_RATIO and tau != 1e-3:
+        pytest.skip("tau does not enter Eq. 1")
+    cfg = dataclasses.replace(synth.CONFIGS["P4"], name=f"P4-{tau}", B=2, tau=tau, accept_mode=accept_mode,
+                              resample_mode=binding.RESAMPLE_TARGET_ALL if accept_mode == binding.ACCEPT_THRESHOLD
+                              else binding.RESAMPLE_MIXED)
+    p = binding.params_from_config(cfg)
+    assert ctx.round_kernel(p, True) == "full"
+    batch = pu.build_batch(cfg)
+    n0 = ctx.kernel_launches()
+    g = pu.gpu_round(ctx, cfg, batch)
+    assert ctx.kernel_launches() - n0 == 2          # the row kernel and the mask kernel: nothing was redone
+    assert ctx.poll_device_status() == 0
+    o = pu.oracle_images(cfg, batch, [0, 1])
+    pu.check_round(cfg, g, o)
+    assert g["n_reject"].sum() > 0
+
+
+@pytest.mark.parametrize("cfg", [
+    dataclasses.replace(BIG, top_k=0, V=4096, dtype="f32", cfg_scale=0.0, seed=270),
+    dataclasses.replace(BIG, top_k=0, V=2048, seed=271),
+    dataclasses.replace(BIG, top_k=0, V=6144, temperature=0.8, seed=272),                    # three pieces per thread
+    dataclasses.replace(BIG, top_k=0, V=8192, pool_k=64, pool_delta=0.3, seed=273),
+    dataclasses.replace(BIG, top_k=0, V=4096, pool_k=500, pool_delta=0.9, cfg_scale=0.0, seed=274),   # several list tiles
+    dataclasses.replace(BIG, top_k=0, V=4096, r=1, H=6, W=6, seed=275),
+    dataclasses.replace(BIG, top_k=0, V=4096, r=3, H=9, W=9, seed=276),
+    dataclasses.replace(BIG, top_k=0, V=4096, resample_mode=binding.RESAMPLE_RESIDUAL_ALL, seed=277),
+    dataclasses.replace(BIG, top_k=0, V=4096, resample_mode=binding.RESAMPLE_ISOLATED_RESIDUAL, radius=2, seed=278),
+    dataclasses.replace(BIG, top_k=0, V=4096, accept_mode=binding.ACCEPT_THRESHOLD, tau=1e-3, seed=279),  # residual draws under Eq. 5
+], ids=lambda c: f"{c.dtype}-V{c.V}-cfg{c.cfg_scale}-pool{c.pool_k}-r{c.r}-m{c.resample_mode}-a{c.accept_mode}")
+def test_round_resident_rows(ctx, cfg):
+    batch = pu.build_batch(cfg)
+    assert ctx.round_kernel(binding.params_from_config(cfg), cfg.has_uncond) == "full"
+    n0 = ctx.kernel_launches()
+    g = pu.gpu_round(ctx, cfg, batch)
+    assert ctx.kernel_launches() - n0 == 2
+    assert ctx.poll_device_status() == 0
+    o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
+    pu.check_round(cfg, g, o)
+    # the general routines give the same decisions and tokens wherever the oracle did not flag the position
+    ctx.set_general_path_only(True)
+    try:
+        d = pu.gpu_round(ctx, cfg, batch)
+    finally:
+        ctx.set_general_path_only(False)
+    pu.check_round(cfg, d, o)

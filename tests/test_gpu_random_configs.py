@@ -70,12 +70,10 @@ def test_random_rounds(ctx, seed):
         ctx.ensure_workspace(p)
         if how != "none":
             transform(batch, how, scale, step)
-            # the draft tokens must have q > 0 under the new logits: redraw them with the library's sampler
-            ctx.mulo_sample_draft(p, batch["draft_lo"], batch["tok_lo"])
-            torch.cuda.synchronize()
-        n0 = ctx.kernel_launches()
+            # the draft tokens must have q > 0 under the new logits: redraw them (oracle's sampler)
+            pu.redraw_tokens(cfg, batch)
         g = pu.gpu_round(ctx, cfg, batch)
-        fast += ctx.kernel_launches() - n0 == 3
+        fast += ctx.round_kernel(p, cfg.has_uncond) != "general"
         o = pu.oracle_images(cfg, batch, list(range(cfg.B)))
         excused = 0
         for b in range(cfg.B):
