@@ -102,7 +102,7 @@ __device__ __forceinline__ float full_one(const unsigned char* crow, const unsig
 }
 
 template <bool BF16, bool HAS_U>
-__global__ void __launch_bounds__(kFThreads, 2) k_round_full(const __grid_constant__ FullArgs a) {
+__global__ void __launch_bounds__(kFThreads, 3) k_round_full(const __grid_constant__ FullArgs a) {
   constexpr int esz = BF16 ? 2 : 4;
   constexpr int N = 16 / esz;   // ids per 16-byte piece
   extern __shared__ __align__(128) unsigned char dyn[];
@@ -300,57 +300,67 @@ __global__ void __launch_bounds__(kFThreads, 2) k_round_full(const __grid_consta
       int J = 0;
       double cJ = 0.0;
       if (pooling) {
+        // Every thread takes `per` consecutive entries of the neighbour list (at most 8: the list
+        // has at most 2047), so one block scan gives every entry's prefix mass.
         const uint16_t* const row = a.nn + (size_t)tok * P.pool_k;
         const int nb = P.pool_k - 1;
+        const int per = (nb + kFThreads - 1) / kFThreads;
+        const int j0 = tid * per;
         for (int x = tid; x < V / 32; x += kFThreads) bitmap[x] = 0u;
         adj[tid] = 0ull;
-        double carry = 0.0;
-        bool open = true;
-        for (int base = 0; base < nb && open; base += kFThreads) {   // block-uniform
-          const int j = base + tid;
-          double pj = 0.0;
-          if (j < nb) {
-            int id = __ldg(row + j + 1);
+        if (tid == 0) sm.first_bad = nb;
+        float e[8];
+        double mine = 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          e[i] = 0.f;
+          if (i < per && j0 + i < nb) {
+            int id = __ldg(row + j0 + i + 1);
             if (id >= V) {
               atomicOr(a.dev_status, MULO_DEV_BAD_TOKEN);
               id = V - 1;
             }
-            const float z = full_one<BF16, HAS_U>(crow, urow, id, P.cfg_scale, P.invT);
-            pj = (double)ex2f(fmaf(z, kLog2e, c0)) / Z;
+            e[i] = ex2f(fmaf(full_one<BF16, HAS_U>(crow, urow, id, P.cfg_scale, P.invT), kLog2e, c0));
+            mine += (double)e[i];
           }
-          if (tid == 0) sm.first_bad = kFThreads;
-          double bef, inc;
-          const double tile_total = block_scan(pj, bef, inc);   // (its barrier also orders first_bad)
-          const double cj = carry + inc;   // inclusive prefix c_{j+1}
-          if (j < nb && !(cj < P.pool_delta)) atomicMin(&sm.first_bad, tid);
-          __syncthreads();
-          const int first_bad = sm.first_bad;
-          const int tile = nb - base < kFThreads ? nb - base : kFThreads;
-          if (first_bad >= tile) {
-            J = base + tile;
-            if (tid == tile - 1) sm.cJ = cj;
-          } else {
-            J = base + first_bad;
-            open = false;
-            if (first_bad == 0 && tid == 0) sm.cJ = carry;
-            if (first_bad > 0 && tid == first_bad - 1) sm.cJ = cj;
-          }
-          carry += tile_total;
-          __syncthreads();
         }
-        if (J > 0) cJ = sm.cJ;
-        // the pooled ids: out of the map of drawable ids, their weights out of their owners' sums
-        for (int j = tid; j < J; j += kFThreads) {
-          int id = __ldg(row + j + 1);
-          if (id >= V) id = V - 1;
-          const uint32_t bit = 1u << (id & 31);
-          const uint32_t old = atomicOr(&bitmap[id >> 5], bit);
-          if (!(old & bit) && id != tok) {   // (a list may name an id twice, or x~ again)
-            const float z = full_one<BF16, HAS_U>(crow, urow, id, P.cfg_scale, P.invT);
-            atomicAdd(&adj[id / W], __float2ull_rz(ex2f(fmaf(z, kLog2e, c0)) * kFix40));
-          }
+        double bef, inc;
+        block_scan(mine, bef, inc);   // (its barrier also publishes first_bad and the cleared map)
+        // c_j < delta, in units of the partition sum
+        const double limit = P.pool_delta * Z;
+        {
+          double c = bef;
+          int bad = nb;
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (i < per && j0 + i < nb) {
+              c += (double)e[i];
+              if (bad == nb && !(c < limit)) bad = j0 + i;
+            }
+          if (bad < nb) atomicMin(&sm.first_bad, bad);
         }
         __syncthreads();
+        J = sm.first_bad;   // the leading run n_1 .. n_J keeps its prefix mass below delta
+        if (J > 0 && (J - 1) / per == tid) {
+          double c = bef;
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (j0 + i < J) c += (double)e[i];
+          sm.cJ = c / Z;
+        }
+        // the pooled ids: out of the map of drawable ids, their weights out of their owners' sums
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (i < per && j0 + i < J) {
+            int id = __ldg(row + j0 + i + 1);
+            if (id >= V) id = V - 1;
+            const uint32_t bit = 1u << (id & 31);
+            const uint32_t old = atomicOr(&bitmap[id >> 5], bit);
+            if (!(old & bit) && id != tok)   // (a list may name an id twice, or x~ again)
+              atomicAdd(&adj[id / W], __float2ull_rz(e[i] * kFix40));
+          }
+        __syncthreads();
+        if (J > 0) cJ = sm.cJ;
       }
       const double p_tok = sm.p_tok / Z;
       const double mass = p_tok + cJ;   // pooled mass P of Eq. 3
