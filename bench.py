@@ -221,14 +221,12 @@ def run_ours(args, cfg):
     positions = cfg.B * cfg.H * cfg.W
     alg_bytes = cfg.algorithmic_bytes_per_position() * positions
     # inputs that fit the L2 twice over would be served from it on every step after the first: such
-    # workloads get 256 MB written between steps (the write is inside the timed region and is
-    # reported; the row kernel's own time, taken by the library's events, is not affected)
+    # workloads get 256 MB written between steps, and every step is timed by an event pair of its
+    # own so that the writes stay outside the timed regions
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if alg_bytes < 2 * L2_BYTES else None
 
     def step(rnd):
         p.round = rnd
-        if flush is not None:
-            flush.zero_()
         ctx.mulo_round(p, batch["cond"], batch["uncond"], batch["draft_lo"], batch["tok_lo"], batch["nn"],
                        out["out_tok"], out["reject_bits"], out["expand_bits"], None, None, None,
                        out["n_reject"], out["n_expand"], out["first_reject"], stream)
@@ -255,18 +253,27 @@ def run_ours(args, cfg):
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_wall0 = time.time()
-    e0.record(stream)
-    for s in range(K):
-        step(W + s)
-    e1.record(stream)
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for s in range(K):
+            step(W + s)
+        e1.record(stream)
+        pairs = [(e0, e1)]
+    else:
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for s in range(K):
+            flush.zero_()
+            pairs[s][0].record(stream)
+            step(W + s)
+            pairs[s][1].record(stream)
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     t_wall1 = time.time()
-    elapsed_ms = e0.elapsed_time(e1)
+    elapsed_ms = sum(a.elapsed_time(b) for a, b in pairs)
     row_ms, row_n = ctx.read_timing()
     ctx.set_timing(0)
     launches = ctx.kernel_launches() - launches0
@@ -323,7 +330,7 @@ def run_ours(args, cfg):
                        "l2": ("inputs per step (%.2f GB) exceed the 126 MB L2; no flush needed" % (alg_bytes / 1e9)
                               if flush is None else
                               "inputs per step (%.1f MB) would stay in the 126 MB L2: 256 MB written between steps, "
-                              "inside the timed region" % (alg_bytes / 1e6)),
+                              "outside the per-step timed regions" % (alg_bytes / 1e6)),
                        "acceptance_rate": acc, "expected_acceptance_mean_sum_min_p_q": expected_acceptance,
                        "speedup_theoretical_S_T": (cfg.H * cfg.W) / ((1.0 - acc) * cfg.H * cfg.W + cfg.h * cfg.w),
                        "expanded_fraction": n_exp / positions,

@@ -58,7 +58,7 @@ struct FullSmem {
   uint64_t bar_q, bar_t;
   double wtot[2][kFWarps];   // block scans; consecutive scans alternate
   double bd[kFWarps];        // block sums
-  float bf[kFWarps];         // block maxima
+  float bf[2][kFWarps];      // block maxima; consecutive reductions alternate
   uint32_t rnd[3];
   double p_tok, q_tok;       // exp(z - max) of x~ at the current position; q(x~) of the parent
   double cJ;                 // pooled prefix mass c_J
@@ -163,15 +163,17 @@ __global__ void __launch_bounds__(kFThreads, 3) k_round_full(const __grid_consta
   };
 
   // ---- block helpers (every thread gets the result; fixed order)
-  auto block_max_f = [&](float v) -> float {
+  int max_call = 0;
+  auto block_max_f = [&](float v) -> float {   // one barrier: consecutive calls alternate buffers
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(kFull, v, o));
-    if (lane == 0) sm.bf[warp] = v;
+    float* const bf = sm.bf[max_call & 1];
+    ++max_call;
+    if (lane == 0) bf[warp] = v;
     __syncthreads();
-    float t = sm.bf[0];
+    float t = bf[0];
 #pragma unroll
-    for (int w = 1; w < kFWarps; ++w) t = fmaxf(t, sm.bf[w]);
-    __syncthreads();
+    for (int w = 1; w < kFWarps; ++w) t = fmaxf(t, bf[w]);
     return t;
   };
   int scan_call = 0;
@@ -435,20 +437,33 @@ __global__ void __launch_bounds__(kFThreads, 3) k_round_full(const __grid_consta
           continue;
         }
         const double y = u * total;
-        if (bef <= y && y < inc) {   // this thread owns u * total: walk its ids in ascending order
+        // One thread owns u * total; its WARP walks that thread's ids together, 32 at a time in
+        // ascending order: weights, an inclusive scan in double, the first id whose running sum
+        // passes y.
+        const unsigned owner_mask = __ballot_sync(kFull, bef <= y && y < inc);
+        if (owner_mask) {   // warp-uniform
+          const int src = __ffs(owner_mask) - 1;
+          const int o_id0 = __shfl_sync(kFull, id0, src);
+          double c = __shfl_sync(kFull, bef, src);
           int pick = -1, last_pos = -1;
-          double c = bef;
-          for (int x = id0; x < id0 + W && pick < 0; ++x) {
-            const float w = weight(x, resid);
-            if (w > 0.f) {
-              c += (double)w;
-              last_pos = x;
-              if (c > y) pick = x;
+          for (int x0 = o_id0; x0 < o_id0 + W && pick < 0; x0 += 32) {
+            const int x = x0 + lane;
+            const float w = x < o_id0 + W ? weight(x, resid) : 0.f;
+            double run = (double)w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const double n = __shfl_up_sync(kFull, run, o);
+              if (lane >= o) run += n;
             }
+            const unsigned has = __ballot_sync(kFull, w > 0.f);
+            const unsigned hit = __ballot_sync(kFull, w > 0.f && c + run > y);
+            if (has) last_pos = x0 + 31 - __clz(has);
+            if (hit) pick = x0 + __ffs(hit) - 1;
+            c += __shfl_sync(kFull, run, 31);
           }
           // (rounding left the walk short of y: the last id with weight; none at all cannot be,
-          // the thread's sum being positive -- then x~ or the first id stands in)
-          *out = pick >= 0 ? pick : last_pos >= 0 ? last_pos : id0;
+          // the thread's sum being positive -- then the thread's first id stands in)
+          if (lane == 0) *out = pick >= 0 ? pick : last_pos >= 0 ? last_pos : o_id0;
         }
         pending &= ~(is_res ? kDrawResidual : kDrawTarget);
         no_mass = false;
