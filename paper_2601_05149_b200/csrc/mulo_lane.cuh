@@ -1066,39 +1066,49 @@ __global__ void __launch_bounds__(kLThreads, 3)
         }
         const double y = u * total;
         const double lo = before + excl, hi = before + inc;
-        if (lo <= y && y < hi) {
-          // this thread owns u * total: walk its entries with the same arithmetic and order
-          int pick = -1, last_pos = -1;
-          float acc = 0.f;
-#pragma unroll 1
-          for (int hf = 0; hf < 2 && pick < 0; ++hf) {
-            uint32_t m = hf ? m_hi : m_lo;
-            const uint32_t dm = hf ? dm_hi : dm_lo;
-            uint32_t ad = hf ? t_base + (uint32_t)(n_lo * step) : t_base;
-            const uint32_t qb = hf ? q_base + (uint32_t)(nq_lo * step) : q_base;
-            const int id0 = tid * W + 32 * hf;
-            while (m && pick < 0) {
-              const uint32_t bit = m & (0u - m);
-              m ^= bit;
-              const float z = lds_f32(ad);
-              ad += step;
-              float w = ex2f(fmaf(z, kLog2e, c0));
-              if (resid) {
-                w = __fmul_rn(w, invZp);
-                if (dm & bit) w = fmaxf(__fsub_rn(w, lds_f32(qb + (uint32_t)(__popc(dm & (bit - 1u)) * step))), 0.f);
-              }
-              if (z >= theta && w > 0.f) {
-                acc += w;
-                last_pos = id0 + __ffs(bit) - 1;
-                if (lo + (double)acc > y) pick = last_pos;
+        // One thread owns u * total; its WARP walks that thread's entries together: lane k takes the
+        // owner's k-th entry (a thread holds at most 32), finds the entry's id by the k-th set bit of
+        // the owner's mask, forms its weight, and an inclusive scan in double finds the first entry
+        // whose running sum passes y.
+        const unsigned own = __ballot_sync(kFull, lo <= y && y < hi);
+        if (own) {   // warp-uniform
+          const int src = __ffs(own) - 1;
+          const uint32_t o_mlo = __shfl_sync(kFull, m_lo, src), o_mhi = __shfl_sync(kFull, m_hi, src);
+          const uint32_t o_dlo = __shfl_sync(kFull, dm_lo, src), o_dhi = __shfl_sync(kFull, dm_hi, src);
+          const uint32_t o_tb = __shfl_sync(kFull, t_base, src), o_qb = __shfl_sync(kFull, q_base, src);
+          const double o_lo = __shfl_sync(kFull, lo, src);
+          const int o_nlo = __popc(o_mlo), o_n = o_nlo + __popc(o_mhi);
+          const bool have = lane < o_n, upper = lane >= o_nlo;
+          const uint32_t mm = upper ? o_mhi : o_mlo, dd = upper ? o_dhi : o_dlo;
+          const int pos = have ? (int)__fns(mm, 0u, (upper ? lane - o_nlo : lane) + 1) : 0;
+          const uint32_t bit = 1u << pos;
+          float w = 0.f;
+          if (have) {
+            const float z = lds_f32(o_tb + (uint32_t)(lane * step));
+            w = ex2f(fmaf(z, kLog2e, c0));
+            if (resid) {
+              w = __fmul_rn(w, invZp);
+              if (dd & bit) {
+                const int qi = (upper ? __popc(o_dlo) : 0) + __popc(dd & (bit - 1u));
+                w = fmaxf(__fsub_rn(w, lds_f32(o_qb + (uint32_t)(qi * step))), 0.f);
               }
             }
+            if (!(z >= theta)) w = 0.f;
           }
-          // rounding left the sum short: the last id with weight.  No id with weight at all: the
-          // thread's sum was rounding noise of the difference above (about once in 1e8 draws) --
+          double run = (double)w;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const double v = __shfl_up_sync(kFull, run, o);
+            if (lane >= o) run += v;
+          }
+          const unsigned has = __ballot_sync(kFull, w > 0.f);
+          const unsigned hit = __ballot_sync(kFull, w > 0.f && o_lo + run > y);
+          // rounding left the sum short: the last entry with weight.  No entry with weight at all:
+          // the thread's sum was rounding noise of the difference above (about once in 1e8 draws) --
           // the position goes to the general routines
-          *out = pick >= 0 ? pick : last_pos;
-          if (pick < 0 && last_pos < 0) {
+          const int chosen = hit ? __ffs(hit) - 1 : has ? 31 - __clz(has) : -1;
+          if (lane == chosen) *out = ((tid & ~31) + src) * W + (upper ? 32 : 0) + pos;
+          if (chosen < 0 && lane == 0) {
             atomicOr(a.dev_status, MULO_DEV_DENSE_FALLBACK);
             defer(g);
           }
