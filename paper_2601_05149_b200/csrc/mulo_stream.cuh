@@ -932,7 +932,21 @@ __global__ void __launch_bounds__(kSThreads, 3) k_round_stream(const __grid_cons
       if (keep) {
         const float e = IS_Q ? qval[at] : __uint_as_float(cand[at].x);
         z += (double)e;
-        if (own && (!IS_Q || SAMPLE)) atomicAdd(&seg_c[seg], e);
+        if (own && (!IS_Q || SAMPLE)) {
+          // The set-aside slots were handed out in no fixed order.  So that the segment sum does not
+          // depend on it, the kept member with the lowest candidate index of a segment adds ALL the
+          // segment's kept members at once, summed in double (exact: entries of one histogram bin
+          // share their exponent or differ by one).
+          bool leader = true;
+          double all = 0.0;
+          for (int j = 0; j < mcount; ++j)
+            if (rs.member_seg[j] == seg && rs.member_z[j] >= th) {
+              const int aj = rs.member_at[j];
+              leader = leader && aj >= at;
+              all += (double)(IS_Q ? qval[aj] : __uint_as_float(cand[aj].x));
+            }
+          if (leader) seg_c[seg] = (float)((double)seg_c[seg] + all);
+        }
       } else if (own) {
         if (IS_Q) qval[at] = 0.f;
         else cand[at].x = 0u;

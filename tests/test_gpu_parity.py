@@ -481,11 +481,16 @@ def test_draft_token_without_draft_mass(ctx, fast):
                 assert g["reject"][b, y, x] == (0 if o[b]["p_tok"][y, x] > 0 else 1)
 
 
-def test_round_is_bit_reproducible_at_launch_size(ctx):
-    """The benchmark's workload (B = 32): the same call twice, and once more from another stream,
-    gives every output array bit for bit -- decisions depend on (seed, image, position, round) and the
-    inputs only, not on how CTAs were scheduled."""
-    cfg = synth.CONFIGS["C4"]
+@pytest.mark.parametrize("name", ["C4", "C2x8", "P4x4"])
+def test_round_is_bit_reproducible_at_launch_size(ctx, name):
+    """The benchmark's workload (B = 32) on the lane kernel, a pooled top-k workload on the streaming
+    kernel and the paper-default workload on the resident-row kernel: the same call twice, and once
+    more from another stream, gives every output array bit for bit -- decisions depend on (seed,
+    image, position, round) and the inputs only, not on how CTAs were scheduled."""
+    cfg = {"C4": synth.CONFIGS["C4"], "C2x8": dataclasses.replace(synth.CONFIGS["C2"], B=8),
+           "P4x4": dataclasses.replace(synth.CONFIGS["P4"], B=4)}[name]
+    assert ctx.round_kernel(binding.params_from_config(cfg), cfg.has_uncond) == \
+        {"C4": "lane", "C2x8": "stream", "P4x4": "full"}[name]
     batch = pu.build_batch(cfg, images=[])      # nothing here goes to the oracle
     p = binding.params_from_config(cfg)
     ctx.ensure_workspace(p)
