@@ -87,6 +87,29 @@ __device__ __forceinline__ void full_piece(uint32_t ac, uint32_t au, float s, fl
     }
   }
 }
+// The same piece as pairs of ids, with packed fp32 instructions (each half one IEEE rounding, as the
+// definition of a pre-processed logit requires: d = c - u; v = fma(s, d, u); z = v * invT)
+template <bool BF16, bool ROW_U, bool SCALE>
+__device__ __forceinline__ void full_piece2(uint32_t ac, uint32_t au, float2 s2, float2 t2, float2 (&z)[BF16 ? 4 : 2]) {
+  const uint4 c = lds128(ac);
+  uint4 u = make_uint4(0, 0, 0, 0);
+  if (ROW_U) u = lds128(au);
+  const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, uw[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int j = 0; j < (BF16 ? 4 : 2); ++j) {
+    float2 v, un;
+    if (BF16) {
+      v = make_float2(bf16_lo(cw[j]), bf16_hi(cw[j]));
+      un = make_float2(bf16_lo(uw[j]), bf16_hi(uw[j]));
+    } else {
+      v = make_float2(__uint_as_float(cw[2 * j]), __uint_as_float(cw[2 * j + 1]));
+      un = make_float2(__uint_as_float(uw[2 * j]), __uint_as_float(uw[2 * j + 1]));
+    }
+    if (ROW_U) v = __ffma2_rn(s2, __ffma2_rn(un, make_float2(-1.f, -1.f), v), un);   // fma(u, -1, c) rounds as c - u
+    if (SCALE) v = __fmul2_rn(v, t2);
+    z[j] = v;
+  }
+}
 // z of one id of a resident row
 template <bool BF16, bool ROW_U>
 __device__ __forceinline__ float full_one(const unsigned char* crow, const unsigned char* urow, int x, float s, float invT) {
@@ -207,27 +230,41 @@ __global__ void __launch_bounds__(kFThreads, 3) k_round_full(const __grid_consta
 
   // ---- one pass over this thread's part of a resident row: running maximum m and the sum of
   //      2^((z - m) log2 e) against it
-  auto softmax_pass = [&](auto row_u_tag, uint32_t at_c, uint32_t at_u, float s, float& m, float& sum) {
+  auto softmax_pass_t = [&](auto row_u_tag, auto scale_tag, uint32_t at_c, uint32_t at_u, float s, float& m, float& sum) {
     constexpr bool ROW_U = decltype(row_u_tag)::value;
+    constexpr bool SCALE = decltype(scale_tag)::value;
+    constexpr int NP = N / 2;   // pairs per piece
+    const float2 s2 = make_float2(s, s), t2 = make_float2(P.invT, P.invT), l2 = make_float2(kLog2e, kLog2e);
     m = -INFINITY;
-    sum = 0.f;
+    float2 acc = make_float2(0.f, 0.f);
     int ci = start;
 #pragma unroll 1
     for (int i = 0; i < nch; ++i) {
-      float z[N];
-      full_piece<BF16, ROW_U>(at_c + (uint32_t)ci * 16u, at_u + (uint32_t)ci * 16u, s, P.invT, z);
+      float2 z[NP];
+      full_piece2<BF16, ROW_U, SCALE>(at_c + (uint32_t)ci * 16u, at_u + (uint32_t)ci * 16u, s2, t2, z);
       if (++ci == nch) ci = 0;
-      float cm = z[0];
+      float cm = fmaxf(z[0].x, z[0].y);
 #pragma unroll
-      for (int j = 1; j < N; ++j) cm = fmaxf(cm, z[j]);
+      for (int j = 1; j < NP; ++j) cm = fmaxf(cm, fmaxf(z[j].x, z[j].y));
       if (cm > m) {
-        sum *= ex2f((m - cm) * kLog2e);   // (0 * 2^-inf = 0 on the first piece)
+        const float f = ex2f((m - cm) * kLog2e);   // (0 * 2^-inf = 0 on the first piece)
+        acc = __fmul2_rn(acc, make_float2(f, f));
         m = cm;
       }
       const float c0 = -m * kLog2e;
+      const float2 c2 = make_float2(c0, c0);
 #pragma unroll
-      for (int j = 0; j < N; ++j) sum += ex2f(fmaf(z[j], kLog2e, c0));
+      for (int j = 0; j < NP; ++j) {
+        const float2 t = __ffma2_rn(z[j], l2, c2);
+        acc = __fadd2_rn(acc, make_float2(ex2f(t.x), ex2f(t.y)));
+      }
     }
+    sum = acc.x + acc.y;
+  };
+  const bool scale = P.invT != 1.0f;
+  auto softmax_pass = [&](auto row_u_tag, uint32_t at_c, uint32_t at_u, float s, float& m, float& sum) {
+    if (scale) softmax_pass_t(row_u_tag, std::true_type{}, at_c, at_u, s, m, sum);   // block-uniform
+    else softmax_pass_t(row_u_tag, std::false_type{}, at_c, at_u, s, m, sum);
   };
 
   for (int parent = p_begin; parent < p_end; ++parent) {
