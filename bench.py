@@ -38,7 +38,7 @@ UNIT = "positions/s"
 # its kernel changes, and the line then reports null until the counters have been taken again.
 TRAFFIC_BYTES_PER_POSITION = {
     ("C4", "lane"): 74268.0,   # 608.4 MB per launch of 8192 positions (algorithmic: 73,752 B per position)
-    ("P4", "full"): 66590.0,   # 545.5 MB per launch of 8192 positions (algorithmic: 67,560 B; the lists come from L2)
+    ("P4", "full"): 66598.0,   # 545.6 MB per launch of 8192 positions (algorithmic: 67,560 B; the lists come from L2)
 }
 L2_BYTES = 126 << 20
 
